@@ -1,0 +1,206 @@
+/*
+ * libdiloco - the DiLoCo outer-optimisation step (standard, naive delayed, eager) and the
+ * inner AdamW step as fused sm_100a CUDA kernels, behind a plain C ABI.
+ *
+ * Method: "Eager Updates For Overlapped Communication and Computation in DiLoCo",
+ * Section 2, Algorithms 1-3.  M workers are simulated as M replica parameter buffers on ONE
+ * GPU; the cross-worker all-reduce of the outer gradients (line 8 of each algorithm) is
+ * replaced by a fixed-order reduction over the replica axis inside the kernel, and the
+ * one-phase delay of its result ("async-send" / "block-receive") by a state buffer that is
+ * written at outer step k and read at outer step k+1.
+ *
+ * Notation (the paper's): M replicas, H inner steps per outer step, theta_m the current
+ * parameters of replica m, s_m = theta_m^(t-H) its start-of-phase ("outer") parameters,
+ * Delta_m = s_m - theta_m the local outer gradient, Delta = (1/M) sum_m Delta_m the
+ * all-reduced one, b_m the momentum buffer of OuterOpt (SGD with Nesterov momentum),
+ * eta / mu the outer learning rate / momentum.  InnerOpt is AdamW.
+ *
+ * General rules of this ABI
+ *   - every pointer inside diloco_buffers_t is a DEVICE pointer on the device that is
+ *     current when diloco_state_init is called; the memory is BORROWED: the caller
+ *     allocates it, keeps it alive while the state exists and frees it afterwards.  The
+ *     library never allocates or frees device memory.
+ *   - every other pointer (config, buffers struct, out-parameters) is a HOST pointer.
+ *   - layout: every [M, stride] buffer is replica-major, element (m, i) at m*stride + i,
+ *     0 <= i < P <= stride.  Elements with i >= P are padding: never read, never written.
+ *     stride * sizeof(element) must be a multiple of 128 bytes for every buffer (so stride
+ *     is a multiple of 64 when any buffer is bf16, else of 32), base pointers 16-byte
+ *     aligned.  grads use their own stride with the same rule.
+ *   - all kernels are launched asynchronously on the stream the caller passes
+ *     (a cudaStream_t cast to void*; NULL = the legacy default stream).  No call
+ *     synchronises the device.  All buffers are updated in place.
+ *   - every call returns a status (0 = DILOCO_OK, negative = error); nothing throws or
+ *     aborts.  On error nothing has been launched and the state is unchanged.
+ *   - arithmetic: fp32, one IEEE round-to-nearest-even per operation, no FMA contraction,
+ *     IEEE division and square root; the sum over replicas runs m = 0 .. M-1 in order; 1/M
+ *     is a division by (float)M.  bf16 is a storage type only (round-to-nearest-even).
+ *   - a state is not thread-safe: one caller at a time.
+ */
+#ifndef DILOCO_H_
+#define DILOCO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DILOCO_MAX_M 64
+
+enum {
+  DILOCO_OK = 0,
+  DILOCO_ERR_INVALID_ARG = -1,    /* null pointer, M < 1, P < 1, stride < P, bad dtype, bad hyper-parameter */
+  DILOCO_ERR_MISALIGNED = -2,     /* base pointer not 16-byte aligned or stride bytes not a multiple of 128 */
+  DILOCO_ERR_BAD_STATE = -3,      /* the state lacks a buffer this call needs */
+  DILOCO_ERR_CUDA = -4,           /* a CUDA runtime call failed; see diloco_last_cuda_error */
+  DILOCO_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait ran out (see diloco_check_device_status) */
+  DILOCO_ERR_UNSUPPORTED = -6     /* M > DILOCO_MAX_M or a size beyond a fixed limit */
+};
+
+/* storage of theta */
+enum {
+  DILOCO_THETA_F32 = 0,        /* theta is fp32 */
+  DILOCO_THETA_BF16 = 1,       /* theta is bf16; Delta_m is formed from the stored (rounded) value */
+  DILOCO_THETA_MASTER_BF16 = 2 /* fp32 master (the value) + bf16 working copy written alongside */
+};
+enum { DILOCO_GRAD_F32 = 0, DILOCO_GRAD_BF16 = 1 };
+
+/* kernel implementation selector (performance only; results are bit-identical) */
+enum {
+  DILOCO_IMPL_AUTO = 0,
+  DILOCO_IMPL_DIRECT = 1, /* register-resident columns, 128-bit global loads and stores */
+  DILOCO_IMPL_BULK = 2    /* replica tiles staged through shared memory by the TMA unit (1-D bulk copies) */
+};
+
+typedef struct {
+  int32_t M;            /* number of replicas (Alg. 1-3 "Require M replicas") */
+  int32_t H;            /* inner steps per outer step (Alg. 1-3 "Synchronization frequency H"); bookkeeping only */
+  int64_t P;            /* flat parameters per replica */
+  int64_t stride;       /* elements between consecutive replicas in every [M, stride] state buffer */
+  float outer_lr;       /* eta  of OuterOpt (Section 3: tuned to 0.4 in the paper) */
+  float outer_momentum; /* mu   of OuterOpt, in [0, 1) */
+  float beta1, beta2;   /* AdamW, each in [0, 1) */
+  float eps;            /* AdamW, >= 0, added after the square root */
+  float weight_decay;   /* AdamW, decoupled, >= 0 */
+  int32_t theta_kind;   /* DILOCO_THETA_* */
+  int32_t grad_kind;    /* DILOCO_GRAD_* : dtype of the grads argument of diloco_inner_adamw */
+  int32_t have_prev;    /* 1: delta_prev_local / delta_prev_avg already hold the previous phase's
+                           gradients (t > H); 0: the next delayed / eager call is the first outer step */
+  int32_t impl;         /* DILOCO_IMPL_* */
+} diloco_config_t;
+
+typedef struct {
+  void *theta;             /* [M, stride] fp32 or bf16 per theta_kind: theta_m^(t)                      */
+  float *master;           /* [M, stride] fp32, only for DILOCO_THETA_MASTER_BF16, else NULL            */
+  float *start;            /* [M, stride] fp32: s_m = theta_m^(t-H)                 (Alg. 1-3 line 7)   */
+  float *delta_prev_local; /* [M, stride] fp32: Delta_m^(t-H); eager only, else may be NULL (Alg. 3 l.11) */
+  float *delta_prev_avg;   /* [stride]    fp32: Delta^(t-H), the all-reduce in flight; delayed and eager,
+                              may be NULL if only the standard step is used         (Alg. 2-3 line 10)  */
+  float *outer_mom;        /* [M, stride] fp32: b_m, Nesterov buffer of OuterOpt                        */
+  float *adam_m;           /* [M, stride] fp32 first moment;  NULL if diloco_inner_adamw is not used    */
+  float *adam_v;           /* [M, stride] fp32 second moment; NULL if diloco_inner_adamw is not used    */
+  uint32_t *device_status; /* 1 word, zero-initialised by the caller; needed only by DILOCO_IMPL_BULK,
+                              whose bounded mbarrier waits record a give-up here; else may be NULL      */
+} diloco_buffers_t;
+
+typedef struct diloco_state diloco_state_t; /* opaque, host memory, owned by the library */
+
+/*
+ * Create a state handle: validates config and buffers (ranges, alignment), records the
+ * current device and its SM count.  *out is set only on success.  Launches nothing.
+ * Errors: INVALID_ARG, MISALIGNED, UNSUPPORTED, CUDA (no usable device).
+ */
+int diloco_state_init(const diloco_config_t *config, const diloco_buffers_t *buffers, diloco_state_t **out);
+
+/* Free the host handle.  Device buffers are the caller's and are not touched.  NULL is OK. */
+int diloco_state_free(diloco_state_t *state);
+
+/*
+ * Inner optimisation step, Alg. 1-3 line 5 with InnerOpt = AdamW, for all M replicas in one
+ * launch: with k = the state's inner-step counter + 1,
+ *     m <- beta1 m + (1-beta1) g,  v <- beta2 v + ((1-beta2) g) g,
+ *     theta <- theta - lr * ( (m/(1-beta1^k)) / (sqrt(v/(1-beta2^k)) + eps) + weight_decay * theta ).
+ * grads: device pointer, [M, grad_stride] of config.grad_kind, read only.  lr: this step's
+ * inner learning rate (the schedule is the caller's).  The bias corrections are computed on
+ * the host in double and rounded to fp32.  Increments the inner-step counter on success.
+ * Errors: INVALID_ARG, MISALIGNED, BAD_STATE (no Adam moments), CUDA.
+ */
+int diloco_inner_adamw(diloco_state_t *state, const void *grads, int64_t grad_stride, float lr, void *cuda_stream);
+
+/*
+ * Outer step of standard DiLoCo, Algorithm 1 lines 7-10, one fused pass:
+ *     Delta_m = s_m - theta_m;  Delta = (1/M) sum_m Delta_m;
+ *     b_m <- mu b_m + Delta;  s_m <- s_m - eta (Delta + mu b_m);  theta_m <- s_m.
+ * Touches theta (master), start, outer_mom only.
+ */
+int diloco_outer_standard(diloco_state_t *state, void *cuda_stream);
+
+/*
+ * Outer step with naive delayed outer gradients, Algorithm 2 lines 7-11: as above but
+ * OuterOpt consumes delta_prev_avg (the mean formed at the previous outer step), and the new
+ * mean replaces it afterwards.  If have_prev == 0 (t = H) nothing is applied: the mean is
+ * recorded, s_m <- theta_m, theta and outer_mom are unchanged, have_prev becomes 1.
+ * Errors additionally: BAD_STATE (delta_prev_avg missing).
+ */
+int diloco_outer_delayed(diloco_state_t *state, void *cuda_stream);
+
+/*
+ * Outer step with eager updates, Algorithm 3 lines 7-12, one fused pass:
+ *     Delta_m = s_m - theta_m;  Delta = (1/M) sum_m Delta_m;
+ *     g_m = (Delta_m - delta_prev_local_m) / M + delta_prev_avg          (line 11)
+ *     b_m <- mu b_m + g_m;  s_m <- s_m - eta (g_m + mu b_m);  theta_m <- s_m  (line 12)
+ *     delta_prev_local_m <- Delta_m;  delta_prev_avg <- Delta.
+ * have_prev == 0: first outer step, as for diloco_outer_delayed, also recording Delta_m.
+ * Errors additionally: BAD_STATE (delta_prev_local or delta_prev_avg missing).
+ */
+int diloco_outer_eager(diloco_state_t *state, void *cuda_stream);
+
+/*
+ * The same three steps restricted to parameter indices [offset, offset + len) of every
+ * replica (a fragment, as Streaming DiLoCo applies the outer step to parts of the model
+ * on different schedules, Section 3).  variant: 0 standard, 1 delayed, 2 eager.  bootstrap
+ * != 0 performs the first-outer-step form for this fragment; the state's have_prev flag and
+ * outer-step counter are NOT consulted or changed: per-fragment bookkeeping is the caller's.
+ * offset must be a multiple of 32 elements (64 if theta is bf16); len >= 1; offset + len <= P.
+ */
+int diloco_outer_fragment(diloco_state_t *state, int32_t variant, int32_t bootstrap,
+                          int64_t offset, int64_t len, void *cuda_stream);
+
+/*
+ * End-to-end form of the three outer steps for callers whose state lives in HOST memory:
+ * copies every state buffer the variant reads from the host_* buffers (same layout and
+ * dtypes as `state`'s device buffers, which serve as the staging area) to the device,
+ * runs the step, and copies every buffer it writes back, chunked along P so that
+ * copies and kernels of different chunks overlap on the three streams given.  host: a
+ * diloco_buffers_t whose pointers are HOST pointers (pinned memory for full copy speed);
+ * streams: three distinct cudaStream_t cast to void* (h2d, compute, d2h); chunk: elements
+ * per chunk, a multiple of 64.  Returns after enqueueing; the caller synchronises streams[2].
+ * Advances have_prev / outer-step counter like the device forms.
+ */
+int diloco_outer_step_host(diloco_state_t *state, int32_t variant, const diloco_buffers_t *host,
+                           void *const streams[3], int64_t chunk);
+
+/* Counters and flags, e.g. for checkpoint / resume (buffers are the caller's to save). */
+int diloco_state_get_counters(const diloco_state_t *state, int64_t *inner_step, int64_t *outer_step, int32_t *have_prev);
+int diloco_state_set_counters(diloco_state_t *state, int64_t inner_step, int64_t outer_step, int32_t have_prev);
+int diloco_set_outer_hparams(diloco_state_t *state, float outer_lr, float outer_momentum);
+int diloco_set_impl(diloco_state_t *state, int32_t impl);
+
+/*
+ * Read the state's device_status word (synchronises the given stream first).  Returns
+ * DILOCO_OK if it is zero or absent, DILOCO_ERR_DEVICE_TIMEOUT if a kernel gave up a bounded
+ * wait (its results are then invalid), DILOCO_ERR_CUDA on a runtime error.
+ */
+int diloco_check_device_status(diloco_state_t *state, void *cuda_stream);
+
+/* Number of kernels this library has launched in this process so far. */
+int64_t diloco_launch_count(void);
+/* The raw cudaError_t of the last failed runtime call made by the library (0 if none). */
+int32_t diloco_last_cuda_error(void);
+/* Static, never NULL. */
+const char *diloco_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DILOCO_H_ */
