@@ -1,0 +1,201 @@
+"""ctypes binding of libdiloco.so: the same names as include/diloco.h, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; this module converts torch
+tensors to device pointers and checks status codes.  There is no fallback: if the shared
+library has not been built (``python -m paper_2502_12996_b200.build``) loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional
+
+PKG = Path(__file__).resolve().parent
+LIB_PATH = PKG / "libdiloco.so"
+
+OK, ERR_INVALID_ARG, ERR_MISALIGNED, ERR_BAD_STATE, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
+THETA_F32, THETA_BF16, THETA_MASTER_BF16 = 0, 1, 2
+GRAD_F32, GRAD_BF16 = 0, 1
+IMPL_AUTO, IMPL_DIRECT, IMPL_BULK = 0, 1, 2
+STANDARD, DELAYED, EAGER = 0, 1, 2
+MAX_M = 64
+
+
+class Config(ctypes.Structure):
+    """diloco_config_t"""
+    _fields_ = [("M", ctypes.c_int32), ("H", ctypes.c_int32), ("P", ctypes.c_int64), ("stride", ctypes.c_int64),
+                ("outer_lr", ctypes.c_float), ("outer_momentum", ctypes.c_float),
+                ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
+                ("weight_decay", ctypes.c_float), ("theta_kind", ctypes.c_int32), ("grad_kind", ctypes.c_int32),
+                ("have_prev", ctypes.c_int32), ("impl", ctypes.c_int32)]
+
+
+class Buffers(ctypes.Structure):
+    """diloco_buffers_t"""
+    _fields_ = [("theta", ctypes.c_void_p), ("master", ctypes.c_void_p), ("start", ctypes.c_void_p),
+                ("delta_prev_local", ctypes.c_void_p), ("delta_prev_avg", ctypes.c_void_p),
+                ("outer_mom", ctypes.c_void_p), ("adam_m", ctypes.c_void_p), ("adam_v", ctypes.c_void_p),
+                ("device_status", ctypes.c_void_p)]
+
+
+class DilocoError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = status_string(status)
+        if status == ERR_CUDA:
+            msg += f" (cudaError {last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [{status}]")
+
+
+_lib = None
+
+SYMBOLS = {
+    "diloco_state_init": (ctypes.c_int, [ctypes.POINTER(Config), ctypes.POINTER(Buffers), ctypes.POINTER(ctypes.c_void_p)]),
+    "diloco_state_free": (ctypes.c_int, [ctypes.c_void_p]),
+    "diloco_inner_adamw": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p]),
+    "diloco_outer_standard": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_outer_delayed": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_outer_eager": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_outer_fragment": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
+    "diloco_outer_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Buffers), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int64]),
+    "diloco_state_get_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)]),
+    "diloco_state_set_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32]),
+    "diloco_set_outer_hparams": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_float, ctypes.c_float]),
+    "diloco_set_impl": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
+    "diloco_check_device_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_launch_count": (ctypes.c_int64, []),
+    "diloco_last_cuda_error": (ctypes.c_int32, []),
+    "diloco_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+}
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libdiloco.so from the package directory; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2502_12996_b200.build` "
+                               "(there is no CPU fallback)")
+        lib = ctypes.CDLL(str(LIB_PATH))
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load_library().diloco_status_string(int(status)).decode()
+
+
+def last_cuda_error() -> int:
+    return int(load_library().diloco_last_cuda_error())
+
+
+def launch_count() -> int:
+    return int(load_library().diloco_launch_count())
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise DilocoError(status, where)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return stream or None
+    return int(stream.cuda_stream)
+
+
+def make_buffers(theta=None, master=None, start=None, delta_prev_local=None, delta_prev_avg=None, outer_mom=None,
+                 adam_m=None, adam_v=None, device_status=None) -> Buffers:
+    return Buffers(_ptr(theta), _ptr(master), _ptr(start), _ptr(delta_prev_local), _ptr(delta_prev_avg),
+                   _ptr(outer_mom), _ptr(adam_m), _ptr(adam_v), _ptr(device_status))
+
+
+class State:
+    """Owns a diloco_state_t handle and keeps the borrowed tensors alive."""
+
+    def __init__(self, *, M, P, stride, theta, start, outer_mom, master=None, delta_prev_local=None,
+                 delta_prev_avg=None, adam_m=None, adam_v=None, device_status=None, H=0, outer_lr=0.7,
+                 outer_momentum=0.9, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1, theta_kind=THETA_F32,
+                 grad_kind=GRAD_F32, have_prev=1, impl=IMPL_AUTO):
+        self._handle = ctypes.c_void_p()
+        self.tensors = dict(theta=theta, master=master, start=start, delta_prev_local=delta_prev_local,
+                            delta_prev_avg=delta_prev_avg, outer_mom=outer_mom, adam_m=adam_m, adam_v=adam_v,
+                            device_status=device_status)
+        self.config = Config(M, H, P, stride, outer_lr, outer_momentum, beta1, beta2, eps, weight_decay,
+                             theta_kind, grad_kind, int(have_prev), impl)
+        self.buffers = make_buffers(**self.tensors)
+        _check(load_library().diloco_state_init(ctypes.byref(self.config), ctypes.byref(self.buffers),
+                                                ctypes.byref(self._handle)), "diloco_state_init")
+
+    @classmethod
+    def from_dict(cls, st: dict, **kw) -> "State":
+        keys = ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom", "adam_m", "adam_v")
+        args = {k: st.get(k) for k in keys}
+        return cls(M=st["M"], P=st["P"], stride=st["stride"], theta_kind=st["theta_kind"], **args, **kw)
+
+    def close(self) -> None:
+        if self._handle:
+            load_library().diloco_state_free(self._handle)
+            self._handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # --- the entry points, same names as the C ABI
+    def inner_adamw(self, grads, lr, stream=None, grad_stride=None) -> None:
+        gs = grads.stride(0) if grad_stride is None else grad_stride
+        _check(load_library().diloco_inner_adamw(self._handle, _ptr(grads), gs, lr, _stream_ptr(stream)),
+               "diloco_inner_adamw")
+
+    def outer_standard(self, stream=None) -> None:
+        _check(load_library().diloco_outer_standard(self._handle, _stream_ptr(stream)), "diloco_outer_standard")
+
+    def outer_delayed(self, stream=None) -> None:
+        _check(load_library().diloco_outer_delayed(self._handle, _stream_ptr(stream)), "diloco_outer_delayed")
+
+    def outer_eager(self, stream=None) -> None:
+        _check(load_library().diloco_outer_eager(self._handle, _stream_ptr(stream)), "diloco_outer_eager")
+
+    def outer(self, variant: int, stream=None) -> None:
+        (self.outer_standard, self.outer_delayed, self.outer_eager)[variant](stream)
+
+    def outer_fragment(self, variant, bootstrap, offset, length, stream=None) -> None:
+        _check(load_library().diloco_outer_fragment(self._handle, variant, int(bool(bootstrap)), offset, length,
+                                                    _stream_ptr(stream)), "diloco_outer_fragment")
+
+    def outer_step_host(self, variant, host: Buffers, streams, chunk) -> None:
+        arr = (ctypes.c_void_p * 3)(*[int(s.cuda_stream) for s in streams])
+        _check(load_library().diloco_outer_step_host(self._handle, variant, ctypes.byref(host), arr, chunk),
+               "diloco_outer_step_host")
+
+    def get_counters(self):
+        a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int32()
+        _check(load_library().diloco_state_get_counters(self._handle, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+               "diloco_state_get_counters")
+        return a.value, b.value, c.value
+
+    def set_counters(self, inner_step, outer_step, have_prev) -> None:
+        _check(load_library().diloco_state_set_counters(self._handle, inner_step, outer_step, int(have_prev)),
+               "diloco_state_set_counters")
+
+    def set_outer_hparams(self, outer_lr, outer_momentum) -> None:
+        _check(load_library().diloco_set_outer_hparams(self._handle, outer_lr, outer_momentum), "diloco_set_outer_hparams")
+
+    def set_impl(self, impl) -> None:
+        _check(load_library().diloco_set_impl(self._handle, impl), "diloco_set_impl")
+
+    def check_device_status(self, stream=None) -> None:
+        _check(load_library().diloco_check_device_status(self._handle, _stream_ptr(stream)), "diloco_check_device_status")

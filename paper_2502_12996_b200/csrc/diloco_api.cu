@@ -1,0 +1,431 @@
+// Host side of libdiloco: the C ABI declared in include/diloco.h.  Validates arguments,
+// keeps the per-state bookkeeping (counters, have_prev) and launches the kernels of
+// diloco_kernels.cuh / diloco_bulk.cuh on the caller's stream.  No device allocation, no
+// device synchronisation (except diloco_check_device_status), no CPU fallback.
+#include "../../include/diloco.h"
+
+#include <atomic>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "diloco_kernels.cuh"
+
+using namespace diloco;
+
+struct diloco_state {
+  diloco_config_t cfg;
+  diloco_buffers_t buf;
+  int device;
+  int sm_count;
+  int64_t inner_step;
+  int64_t outer_step;
+  int32_t have_prev;
+  std::vector<cudaEvent_t> events; // host-path chunk events, created on first use
+  cudaEvent_t last_d2h;
+};
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+std::atomic<int32_t> g_last_cuda_error{0};
+
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error.store((int32_t)e);
+  return DILOCO_ERR_CUDA;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t theta_elt(int32_t kind) { return kind == DILOCO_THETA_F32 ? 4 : 2; }
+
+int validate_config(const diloco_config_t *c) {
+  if (!c) return DILOCO_ERR_INVALID_ARG;
+  if (c->M < 1 || c->P < 1 || c->stride < c->P || c->H < 0) return DILOCO_ERR_INVALID_ARG;
+  if (c->M > DILOCO_MAX_M) return DILOCO_ERR_UNSUPPORTED;
+  if (c->theta_kind < DILOCO_THETA_F32 || c->theta_kind > DILOCO_THETA_MASTER_BF16) return DILOCO_ERR_INVALID_ARG;
+  if (c->grad_kind < DILOCO_GRAD_F32 || c->grad_kind > DILOCO_GRAD_BF16) return DILOCO_ERR_INVALID_ARG;
+  if (c->impl < DILOCO_IMPL_AUTO || c->impl > DILOCO_IMPL_BULK) return DILOCO_ERR_INVALID_ARG;
+  if (!(c->outer_momentum >= 0.f && c->outer_momentum < 1.f)) return DILOCO_ERR_INVALID_ARG;
+  if (!std::isfinite(c->outer_lr)) return DILOCO_ERR_INVALID_ARG;
+  if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f)) return DILOCO_ERR_INVALID_ARG;
+  if (!(c->eps >= 0.f) || !(c->weight_decay >= 0.f)) return DILOCO_ERR_INVALID_ARG;
+  if (c->have_prev != 0 && c->have_prev != 1) return DILOCO_ERR_INVALID_ARG;
+  // 128-byte rows for every dtype in use
+  if ((c->stride * 4) % 128 != 0) return DILOCO_ERR_MISALIGNED;
+  if (c->theta_kind != DILOCO_THETA_F32 && (c->stride * 2) % 128 != 0) return DILOCO_ERR_MISALIGNED;
+  return DILOCO_OK;
+}
+
+int validate_buffers(const diloco_config_t *c, const diloco_buffers_t *b) {
+  if (!b) return DILOCO_ERR_INVALID_ARG;
+  if (!b->theta || !b->start || !b->outer_mom) return DILOCO_ERR_INVALID_ARG;
+  if (c->theta_kind == DILOCO_THETA_MASTER_BF16 && !b->master) return DILOCO_ERR_INVALID_ARG;
+  if ((b->adam_m == nullptr) != (b->adam_v == nullptr)) return DILOCO_ERR_INVALID_ARG;
+  const void *all[] = {b->theta, b->master, b->start, b->delta_prev_local, b->delta_prev_avg,
+                       b->outer_mom, b->adam_m, b->adam_v};
+  for (const void *p : all)
+    if (p && !aligned16(p)) return DILOCO_ERR_MISALIGNED;
+  if (b->device_status && (reinterpret_cast<uintptr_t>(b->device_status) & 3u)) return DILOCO_ERR_MISALIGNED;
+  return DILOCO_OK;
+}
+
+// blocks to launch for `work` columns: a persistent grid of (resident blocks per SM) x SMs
+template <typename K>
+int grid_for(K kernel, const diloco_state *st, long long work, int *grid) {
+  int per_sm = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (per_sm < 1) per_sm = 1;
+  long long need = (work + kThreads - 1) / kThreads;
+  long long cap = (long long)per_sm * st->sm_count;
+  if (need < 1) need = 1;
+  *grid = (int)(need < cap ? need : cap);
+  return DILOCO_OK;
+}
+
+template <int M, int VAR, int TK, bool BOOT, int V, int MINB>
+int launch_outer_t(const diloco_state *st, const OuterArgs &a, cudaStream_t s) {
+  auto k = outer_step_kernel<M, VAR, TK, BOOT, V, MINB>;
+  int grid = 1;
+  int rc = grid_for(k, st, (a.P + V - 1) / V, &grid);
+  if (rc != DILOCO_OK) return rc;
+  k<<<grid, kThreads, 0, s>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1);
+  return DILOCO_OK;
+}
+
+template <int M, int V, int MINB>
+int launch_outer_m(const diloco_state *st, int var, int tk, bool boot, const OuterArgs &a, cudaStream_t s) {
+#define DILOCO_CASE(VAR_, TK_)                                                            \
+  if (var == VAR_ && tk == TK_) {                                                         \
+    if (VAR_ != VAR_STANDARD && boot) return launch_outer_t<M, VAR_, TK_, true, V, MINB>(st, a, s); \
+    return launch_outer_t<M, VAR_, TK_, false, V, MINB>(st, a, s);                         \
+  }
+  DILOCO_CASE(VAR_STANDARD, TK_F32)
+  DILOCO_CASE(VAR_STANDARD, TK_BF16)
+  DILOCO_CASE(VAR_STANDARD, TK_MASTER_BF16)
+  DILOCO_CASE(VAR_DELAYED, TK_F32)
+  DILOCO_CASE(VAR_DELAYED, TK_BF16)
+  DILOCO_CASE(VAR_DELAYED, TK_MASTER_BF16)
+  DILOCO_CASE(VAR_EAGER, TK_F32)
+  DILOCO_CASE(VAR_EAGER, TK_BF16)
+  DILOCO_CASE(VAR_EAGER, TK_MASTER_BF16)
+#undef DILOCO_CASE
+  return DILOCO_ERR_INVALID_ARG;
+}
+
+int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterArgs &a, cudaStream_t s) {
+  const int tk = st->cfg.theta_kind;
+  switch (st->cfg.M) {
+    case 1: return launch_outer_m<1, 4, 4>(st, var, tk, boot, a, s);
+    case 2: return launch_outer_m<2, 4, 3>(st, var, tk, boot, a, s);
+    case 3: return launch_outer_m<3, 4, 2>(st, var, tk, boot, a, s);
+    case 4: return launch_outer_m<4, 4, 2>(st, var, tk, boot, a, s);
+    case 8: return launch_outer_m<8, 4, 1>(st, var, tk, boot, a, s);
+    case 16: return launch_outer_m<16, 2, 1>(st, var, tk, boot, a, s);
+    default: return launch_outer_m<0, 4, 2>(st, var, tk, boot, a, s);
+  }
+}
+
+// variant-specific buffer requirements
+int check_variant(const diloco_state *st, int var) {
+  if (var < VAR_STANDARD || var > VAR_EAGER) return DILOCO_ERR_INVALID_ARG;
+  if (var != VAR_STANDARD && !st->buf.delta_prev_avg) return DILOCO_ERR_BAD_STATE;
+  if (var == VAR_EAGER && !st->buf.delta_prev_local) return DILOCO_ERR_BAD_STATE;
+  return DILOCO_OK;
+}
+
+OuterArgs outer_args(const diloco_state *st, int64_t offset, int64_t len) {
+  OuterArgs a;
+  const diloco_buffers_t &b = st->buf;
+  a.theta = b.theta ? static_cast<char *>(b.theta) + (size_t)offset * theta_elt(st->cfg.theta_kind) : nullptr;
+  a.master = b.master ? b.master + offset : nullptr;
+  a.start = b.start + offset;
+  a.dpl = b.delta_prev_local ? b.delta_prev_local + offset : nullptr;
+  a.dpa = b.delta_prev_avg ? b.delta_prev_avg + offset : nullptr;
+  a.mom = b.outer_mom + offset;
+  a.P = len;
+  a.stride = st->cfg.stride;
+  a.eta = st->cfg.outer_lr;
+  a.mu = st->cfg.outer_momentum;
+  a.fM = (float)st->cfg.M;
+  a.M = st->cfg.M;
+  return a;
+}
+
+int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t len, cudaStream_t s) {
+  OuterArgs a = outer_args(st, offset, len);
+  return launch_outer_direct(st, var, boot, a, s);
+}
+
+int outer_whole(diloco_state *st, int var, void *stream) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  int rc = check_variant(st, var);
+  if (rc != DILOCO_OK) return rc;
+  const bool boot = (var != VAR_STANDARD) && st->have_prev == 0;
+  rc = launch_outer(st, var, boot, 0, st->cfg.P, static_cast<cudaStream_t>(stream));
+  if (rc != DILOCO_OK) return rc;
+  if (var != VAR_STANDARD) st->have_prev = 1;
+  st->outer_step += 1;
+  return DILOCO_OK;
+}
+
+template <int TK, int GK>
+int launch_adamw_t(const diloco_state *st, const AdamArgs &a, cudaStream_t s) {
+  constexpr int V = 4, U = 2;
+  auto k = adamw_kernel<TK, GK, V, U>;
+  int per_sm = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, 0);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (per_sm < 1) per_sm = 1;
+  const int M = st->cfg.M;
+  long long need = ((a.P + V - 1) / V + (long long)kThreads * U - 1) / ((long long)kThreads * U);
+  long long cap = ((long long)per_sm * st->sm_count + M - 1) / M; // resident blocks shared by the M rows
+  if (need < 1) need = 1;
+  if (cap < 1) cap = 1;
+  dim3 grid((unsigned)(need < cap ? need : cap), (unsigned)M);
+  k<<<grid, kThreads, 0, s>>>(a);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1);
+  return DILOCO_OK;
+}
+
+} // namespace
+
+extern "C" {
+
+int diloco_state_init(const diloco_config_t *config, const diloco_buffers_t *buffers, diloco_state_t **out) {
+  if (!out) return DILOCO_ERR_INVALID_ARG;
+  int rc = validate_config(config);
+  if (rc != DILOCO_OK) return rc;
+  rc = validate_buffers(config, buffers);
+  if (rc != DILOCO_OK) return rc;
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  diloco_state *st = new (std::nothrow) diloco_state();
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  st->cfg = *config;
+  st->buf = *buffers;
+  st->device = dev;
+  st->sm_count = sms;
+  st->inner_step = 0;
+  st->outer_step = 0;
+  st->have_prev = config->have_prev;
+  st->last_d2h = nullptr;
+  *out = st;
+  return DILOCO_OK;
+}
+
+int diloco_state_free(diloco_state_t *st) {
+  if (!st) return DILOCO_OK;
+  for (cudaEvent_t ev : st->events) cudaEventDestroy(ev);
+  if (st->last_d2h) cudaEventDestroy(st->last_d2h);
+  delete st;
+  return DILOCO_OK;
+}
+
+int diloco_inner_adamw(diloco_state_t *st, const void *grads, int64_t grad_stride, float lr, void *stream) {
+  if (!st || !grads) return DILOCO_ERR_INVALID_ARG;
+  if (!st->buf.adam_m || !st->buf.adam_v) return DILOCO_ERR_BAD_STATE;
+  if (grad_stride < st->cfg.P || !std::isfinite(lr)) return DILOCO_ERR_INVALID_ARG;
+  const size_t gelt = st->cfg.grad_kind == DILOCO_GRAD_F32 ? 4 : 2;
+  if (!aligned16(grads) || (grad_stride * (int64_t)gelt) % 128 != 0) return DILOCO_ERR_MISALIGNED;
+  const int64_t k = st->inner_step + 1;
+  AdamArgs a;
+  a.theta = st->buf.theta;
+  a.master = st->buf.master;
+  a.grads = grads;
+  a.m = st->buf.adam_m;
+  a.v = st->buf.adam_v;
+  a.P = st->cfg.P;
+  a.stride = st->cfg.stride;
+  a.gstride = grad_stride;
+  a.lr = lr;
+  a.beta1 = st->cfg.beta1;
+  a.beta2 = st->cfg.beta2;
+  a.omb1 = 1.0f - st->cfg.beta1;
+  a.omb2 = 1.0f - st->cfg.beta2;
+  // bias corrections 1 - beta^k: in double, then one rounding to fp32
+  a.c1 = (float)(1.0 - std::pow((double)st->cfg.beta1, (double)k));
+  a.c2 = (float)(1.0 - std::pow((double)st->cfg.beta2, (double)k));
+  a.eps = st->cfg.eps;
+  a.wd = st->cfg.weight_decay;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = DILOCO_ERR_INVALID_ARG;
+  const int tk = st->cfg.theta_kind, gk = st->cfg.grad_kind;
+#define DILOCO_ADAM(TK_, GK_) \
+  if (tk == TK_ && gk == GK_) rc = launch_adamw_t<TK_, GK_>(st, a, s);
+  DILOCO_ADAM(TK_F32, GK_F32)
+  DILOCO_ADAM(TK_F32, GK_BF16)
+  DILOCO_ADAM(TK_BF16, GK_F32)
+  DILOCO_ADAM(TK_BF16, GK_BF16)
+  DILOCO_ADAM(TK_MASTER_BF16, GK_F32)
+  DILOCO_ADAM(TK_MASTER_BF16, GK_BF16)
+#undef DILOCO_ADAM
+  if (rc != DILOCO_OK) return rc;
+  st->inner_step = k;
+  return DILOCO_OK;
+}
+
+int diloco_outer_standard(diloco_state_t *st, void *stream) { return outer_whole(st, VAR_STANDARD, stream); }
+int diloco_outer_delayed(diloco_state_t *st, void *stream) { return outer_whole(st, VAR_DELAYED, stream); }
+int diloco_outer_eager(diloco_state_t *st, void *stream) { return outer_whole(st, VAR_EAGER, stream); }
+
+int diloco_outer_fragment(diloco_state_t *st, int32_t variant, int32_t bootstrap, int64_t offset, int64_t len,
+                          void *stream) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  int rc = check_variant(st, variant);
+  if (rc != DILOCO_OK) return rc;
+  if (variant == VAR_STANDARD && bootstrap) return DILOCO_ERR_INVALID_ARG;
+  if (offset < 0 || len < 1 || offset > st->cfg.P - len) return DILOCO_ERR_INVALID_ARG;
+  const int64_t q = st->cfg.theta_kind == DILOCO_THETA_F32 ? 32 : 64;
+  if (offset % q != 0) return DILOCO_ERR_MISALIGNED;
+  return launch_outer(st, variant, bootstrap != 0, offset, len, static_cast<cudaStream_t>(stream));
+}
+
+int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buffers_t *host, void *const streams[3],
+                           int64_t chunk) {
+  if (!st || !host || !streams) return DILOCO_ERR_INVALID_ARG;
+  int rc = check_variant(st, variant);
+  if (rc != DILOCO_OK) return rc;
+  if (chunk < 64 || chunk % 64 != 0) return DILOCO_ERR_INVALID_ARG;
+  cudaStream_t s_in = static_cast<cudaStream_t>(streams[0]);
+  cudaStream_t s_k = static_cast<cudaStream_t>(streams[1]);
+  cudaStream_t s_out = static_cast<cudaStream_t>(streams[2]);
+  if (s_in == s_k || s_k == s_out || s_in == s_out) return DILOCO_ERR_INVALID_ARG;
+  const diloco_buffers_t &d = st->buf;
+  const bool boot = (variant != VAR_STANDARD) && st->have_prev == 0;
+  const int tk = st->cfg.theta_kind;
+  // which buffers the variant reads (in) and writes (out); rows = M, or 1 for delta_prev_avg
+  struct Leg { void *dev; void *hst; size_t elt; int rows; bool in, out; };
+  const bool master = tk == DILOCO_THETA_MASTER_BF16;
+  Leg legs[6] = {
+      {d.theta, host->theta, theta_elt(tk), st->cfg.M, !master, !boot},
+      {d.master, host->master, 4, st->cfg.M, master, master && !boot},
+      {d.start, host->start, 4, st->cfg.M, true, true},
+      {d.delta_prev_local, host->delta_prev_local, 4, st->cfg.M, variant == VAR_EAGER && !boot, variant == VAR_EAGER},
+      {d.delta_prev_avg, host->delta_prev_avg, 4, 1, variant != VAR_STANDARD && !boot, variant != VAR_STANDARD},
+      {d.outer_mom, host->outer_mom, 4, st->cfg.M, !boot, !boot},
+  };
+  for (const Leg &l : legs)
+    if ((l.in || l.out) && (!l.dev || !l.hst)) return DILOCO_ERR_INVALID_ARG;
+  const int64_t P = st->cfg.P;
+  const size_t nchunks = (size_t)((P + chunk - 1) / chunk);
+  cudaError_t e;
+  while (st->events.size() < 2 * nchunks) {
+    cudaEvent_t ev;
+    e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_fail(e);
+    st->events.push_back(ev);
+  }
+  if (!st->last_d2h) {
+    e = cudaEventCreateWithFlags(&st->last_d2h, cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_fail(e);
+  } else {
+    // the staging area is reused: do not overwrite it before the previous call has drained
+    e = cudaStreamWaitEvent(s_in, st->last_d2h, 0);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  const size_t row = (size_t)st->cfg.stride;
+  for (size_t c = 0; c < nchunks; ++c) {
+    const int64_t off = (int64_t)c * chunk;
+    const int64_t len = (off + chunk <= P) ? chunk : (P - off);
+    for (const Leg &l : legs) {
+      if (!l.in) continue;
+      e = cudaMemcpy2DAsync(static_cast<char *>(l.dev) + (size_t)off * l.elt, row * l.elt,
+                            static_cast<const char *>(l.hst) + (size_t)off * l.elt, row * l.elt,
+                            (size_t)len * l.elt, (size_t)l.rows, cudaMemcpyHostToDevice, s_in);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+    e = cudaEventRecord(st->events[2 * c], s_in);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamWaitEvent(s_k, st->events[2 * c], 0);
+    if (e != cudaSuccess) return cuda_fail(e);
+    rc = launch_outer(st, variant, boot, off, len, s_k);
+    if (rc != DILOCO_OK) return rc;
+    e = cudaEventRecord(st->events[2 * c + 1], s_k);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamWaitEvent(s_out, st->events[2 * c + 1], 0);
+    if (e != cudaSuccess) return cuda_fail(e);
+    for (const Leg &l : legs) {
+      if (!l.out) continue;
+      e = cudaMemcpy2DAsync(static_cast<char *>(l.hst) + (size_t)off * l.elt, row * l.elt,
+                            static_cast<const char *>(l.dev) + (size_t)off * l.elt, row * l.elt,
+                            (size_t)len * l.elt, (size_t)l.rows, cudaMemcpyDeviceToHost, s_out);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+  }
+  e = cudaEventRecord(st->last_d2h, s_out);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (variant != VAR_STANDARD) st->have_prev = 1;
+  st->outer_step += 1;
+  return DILOCO_OK;
+}
+
+int diloco_state_get_counters(const diloco_state_t *st, int64_t *inner_step, int64_t *outer_step, int32_t *have_prev) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  if (inner_step) *inner_step = st->inner_step;
+  if (outer_step) *outer_step = st->outer_step;
+  if (have_prev) *have_prev = st->have_prev;
+  return DILOCO_OK;
+}
+
+int diloco_state_set_counters(diloco_state_t *st, int64_t inner_step, int64_t outer_step, int32_t have_prev) {
+  if (!st || inner_step < 0 || outer_step < 0 || (have_prev != 0 && have_prev != 1)) return DILOCO_ERR_INVALID_ARG;
+  st->inner_step = inner_step;
+  st->outer_step = outer_step;
+  st->have_prev = have_prev;
+  return DILOCO_OK;
+}
+
+int diloco_set_outer_hparams(diloco_state_t *st, float outer_lr, float outer_momentum) {
+  if (!st || !std::isfinite(outer_lr) || !(outer_momentum >= 0.f && outer_momentum < 1.f)) return DILOCO_ERR_INVALID_ARG;
+  st->cfg.outer_lr = outer_lr;
+  st->cfg.outer_momentum = outer_momentum;
+  return DILOCO_OK;
+}
+
+int diloco_set_impl(diloco_state_t *st, int32_t impl) {
+  if (!st || impl < DILOCO_IMPL_AUTO || impl > DILOCO_IMPL_BULK) return DILOCO_ERR_INVALID_ARG;
+  st->cfg.impl = impl;
+  return DILOCO_OK;
+}
+
+int diloco_check_device_status(diloco_state_t *st, void *stream) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  if (!st->buf.device_status) return DILOCO_OK;
+  uint32_t word = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(&word, st->buf.device_status, sizeof(word), cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return word == 0 ? DILOCO_OK : DILOCO_ERR_DEVICE_TIMEOUT;
+}
+
+int64_t diloco_launch_count(void) { return g_launches.load(); }
+int32_t diloco_last_cuda_error(void) { return g_last_cuda_error.load(); }
+
+const char *diloco_status_string(int status) {
+  switch (status) {
+    case DILOCO_OK: return "ok";
+    case DILOCO_ERR_INVALID_ARG: return "invalid argument";
+    case DILOCO_ERR_MISALIGNED: return "misaligned pointer, stride or offset";
+    case DILOCO_ERR_BAD_STATE: return "state lacks a buffer this call needs";
+    case DILOCO_ERR_CUDA: return "CUDA runtime error";
+    case DILOCO_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case DILOCO_ERR_UNSUPPORTED: return "unsupported size";
+    default: return "unknown status";
+  }
+}
+
+} // extern "C"

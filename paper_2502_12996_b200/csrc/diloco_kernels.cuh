@@ -1,0 +1,381 @@
+// Device code of libdiloco: the fused outer step (Algorithms 1-3, lines 7-12) and the inner
+// AdamW step, register-resident "direct" form.  Compiled for sm_100a only, with
+// -fmad=false: every fp32 operation below is one IEEE round-to-nearest operation, written
+// in the order the algorithms state it, so results are bit-identical for any launch shape.
+//
+// Memory behaviour is the whole design (the path is < 1 flop/byte): each state word is read
+// once and written once, with 128-bit accesses that a warp issues as 512 contiguous bytes,
+// all loads of a column issued before its first dependent use so that one thread keeps
+// (4M+1) x 16 bytes in flight, and streaming cache hints since nothing is reused.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace diloco {
+
+enum { VAR_STANDARD = 0, VAR_DELAYED = 1, VAR_EAGER = 2 };
+enum { TK_F32 = 0, TK_BF16 = 1, TK_MASTER_BF16 = 2 };
+enum { GK_F32 = 0, GK_BF16 = 1 };
+
+constexpr int kThreads = 256;
+
+struct OuterArgs {
+  void *theta;     // [M, stride] fp32 or bf16
+  float *master;   // [M, stride] or nullptr
+  float *start;    // [M, stride]
+  float *dpl;      // [M, stride] Delta_m^(t-H) (eager)
+  float *dpa;      // [stride]    Delta^(t-H)   (delayed, eager)
+  float *mom;      // [M, stride] b_m
+  long long P;      // indices [0, P) are processed (pointers already offset for fragments)
+  long long stride; // elements between replicas
+  float eta, mu, fM;
+  int M;            // used by the runtime-M kernel only
+};
+
+struct AdamArgs {
+  void *theta;
+  float *master;
+  const void *grads;
+  float *m, *v;
+  long long P, stride, gstride;
+  float lr, beta1, beta2, omb1, omb2, c1, c2, eps, wd;
+};
+
+// ---------------------------------------------------------------- vector access helpers
+// V consecutive elements starting at an index that is a multiple of V.  Streaming hints:
+// ld.global.cs / st.global.cs (evict-first), the data is touched once per launch.
+template <int V> struct F32Vec;
+template <> struct F32Vec<4> {
+  static __device__ __forceinline__ void load(const float *p, float (&r)[4]) {
+    float4 t = __ldcs(reinterpret_cast<const float4 *>(p));
+    r[0] = t.x; r[1] = t.y; r[2] = t.z; r[3] = t.w;
+  }
+  static __device__ __forceinline__ void load_cached(const float *p, float (&r)[4]) {
+    float4 t = *reinterpret_cast<const float4 *>(p);
+    r[0] = t.x; r[1] = t.y; r[2] = t.z; r[3] = t.w;
+  }
+  static __device__ __forceinline__ void store(float *p, const float (&r)[4]) {
+    __stcs(reinterpret_cast<float4 *>(p), make_float4(r[0], r[1], r[2], r[3]));
+  }
+};
+template <> struct F32Vec<2> {
+  static __device__ __forceinline__ void load(const float *p, float (&r)[2]) {
+    float2 t = __ldcs(reinterpret_cast<const float2 *>(p));
+    r[0] = t.x; r[1] = t.y;
+  }
+  static __device__ __forceinline__ void load_cached(const float *p, float (&r)[2]) {
+    float2 t = *reinterpret_cast<const float2 *>(p);
+    r[0] = t.x; r[1] = t.y;
+  }
+  static __device__ __forceinline__ void store(float *p, const float (&r)[2]) {
+    __stcs(reinterpret_cast<float2 *>(p), make_float2(r[0], r[1]));
+  }
+};
+template <> struct F32Vec<1> {
+  static __device__ __forceinline__ void load(const float *p, float (&r)[1]) { r[0] = __ldcs(p); }
+  static __device__ __forceinline__ void load_cached(const float *p, float (&r)[1]) { r[0] = *p; }
+  static __device__ __forceinline__ void store(float *p, const float (&r)[1]) { __stcs(p, r[0]); }
+};
+
+__device__ __forceinline__ float bf16_bits_to_f32(unsigned short h) { return __uint_as_float(((unsigned)h) << 16); }
+__device__ __forceinline__ unsigned short f32_to_bf16_bits(float f) {
+  return __bfloat16_as_ushort(__float2bfloat16_rn(f)); // round-to-nearest-even
+}
+
+template <int V> struct BF16Vec;
+template <> struct BF16Vec<4> {
+  static __device__ __forceinline__ void load(const unsigned short *p, float (&r)[4], bool cached = false) {
+    uint2 t = cached ? *reinterpret_cast<const uint2 *>(p) : __ldcs(reinterpret_cast<const uint2 *>(p));
+    r[0] = bf16_bits_to_f32(t.x & 0xffffu); r[1] = bf16_bits_to_f32(t.x >> 16);
+    r[2] = bf16_bits_to_f32(t.y & 0xffffu); r[3] = bf16_bits_to_f32(t.y >> 16);
+  }
+  static __device__ __forceinline__ void store(unsigned short *p, const float (&r)[4]) {
+    uint2 t;
+    t.x = (unsigned)f32_to_bf16_bits(r[0]) | ((unsigned)f32_to_bf16_bits(r[1]) << 16);
+    t.y = (unsigned)f32_to_bf16_bits(r[2]) | ((unsigned)f32_to_bf16_bits(r[3]) << 16);
+    __stcs(reinterpret_cast<uint2 *>(p), t);
+  }
+};
+template <> struct BF16Vec<2> {
+  static __device__ __forceinline__ void load(const unsigned short *p, float (&r)[2], bool cached = false) {
+    unsigned t = cached ? *reinterpret_cast<const unsigned *>(p) : __ldcs(reinterpret_cast<const unsigned *>(p));
+    r[0] = bf16_bits_to_f32(t & 0xffffu); r[1] = bf16_bits_to_f32(t >> 16);
+  }
+  static __device__ __forceinline__ void store(unsigned short *p, const float (&r)[2]) {
+    __stcs(reinterpret_cast<unsigned *>(p), (unsigned)f32_to_bf16_bits(r[0]) | ((unsigned)f32_to_bf16_bits(r[1]) << 16));
+  }
+};
+template <> struct BF16Vec<1> {
+  static __device__ __forceinline__ void load(const unsigned short *p, float (&r)[1], bool cached = false) {
+    unsigned short t = cached ? *p : __ldcs(p);
+    r[0] = bf16_bits_to_f32(t);
+  }
+  static __device__ __forceinline__ void store(unsigned short *p, const float (&r)[1]) { __stcs(p, f32_to_bf16_bits(r[0])); }
+};
+
+// theta_m^(t) as the fp32 value the algorithms operate on
+template <int TK, int V>
+__device__ __forceinline__ void load_theta(const OuterArgs &a, long long at, float (&x)[V], bool cached = false) {
+  if (TK == TK_F32) {
+    if (cached) F32Vec<V>::load_cached(reinterpret_cast<const float *>(a.theta) + at, x);
+    else F32Vec<V>::load(reinterpret_cast<const float *>(a.theta) + at, x);
+  } else if (TK == TK_BF16) {
+    BF16Vec<V>::load(reinterpret_cast<const unsigned short *>(a.theta) + at, x, cached);
+  } else {
+    if (cached) F32Vec<V>::load_cached(a.master + at, x);
+    else F32Vec<V>::load(a.master + at, x);
+  }
+}
+template <int TK, int V>
+__device__ __forceinline__ void store_theta(const OuterArgs &a, long long at, const float (&n)[V]) {
+  if (TK == TK_F32) {
+    F32Vec<V>::store(reinterpret_cast<float *>(a.theta) + at, n);
+  } else if (TK == TK_BF16) {
+    BF16Vec<V>::store(reinterpret_cast<unsigned short *>(a.theta) + at, n);
+  } else {
+    F32Vec<V>::store(a.master + at, n);
+    BF16Vec<V>::store(reinterpret_cast<unsigned short *>(a.theta) + at, n);
+  }
+}
+
+// OuterOpt(theta^(t-H), g): SGD with Nesterov momentum.  b <- mu b + g ; s <- s - eta (g + mu b)
+__device__ __forceinline__ void nesterov(float g, float eta, float mu, float &b, float &s) {
+  float nb = mu * b;
+  nb = nb + g;
+  float u = mu * nb;
+  u = g + u;
+  u = eta * u;
+  s = s - u;
+  b = nb;
+}
+
+// ---------------------------------------------------------------- outer step, compile-time M
+// One column = V consecutive parameter indices of all M replicas.
+template <int M, int VAR, int TK, bool BOOT, int V>
+__device__ __forceinline__ void outer_column(const OuterArgs &a, long long i) {
+  float s[M][V], d[M][V];
+  // Alg. 1-3 line 7: Delta_m = theta_m^(t-H) - theta_m^(t)
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+    F32Vec<V>::load(a.start + m * a.stride + i, s[m]);
+    load_theta<TK, V>(a, m * a.stride + i, d[m]);
+  }
+  if constexpr (BOOT) {
+    // first outer step (t = H): record, do not apply
+    float mean[V];
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      float x[V];
+#pragma unroll
+      for (int e = 0; e < V; ++e) {
+        x[e] = d[m][e];
+        d[m][e] = s[m][e] - x[e];
+        mean[e] = (m == 0) ? d[m][e] : mean[e] + d[m][e];
+      }
+      F32Vec<V>::store(a.start + m * a.stride + i, x);
+      if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + m * a.stride + i, d[m]);
+    }
+#pragma unroll
+    for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
+    F32Vec<V>::store(a.dpa + i, mean);
+  } else {
+  float b[M][V], pl[M][V], pa[V];
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+    F32Vec<V>::load(a.mom + m * a.stride + i, b[m]);
+    if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + m * a.stride + i, pl[m]);
+  }
+  if (VAR != VAR_STANDARD) F32Vec<V>::load(a.dpa + i, pa);
+
+  // line 8: Delta = (1/M) sum_m Delta_m, m in order (the all-reduce)
+  float mean[V];
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      d[m][e] = s[m][e] - d[m][e];
+      mean[e] = (m == 0) ? d[m][e] : mean[e] + d[m][e];
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
+
+#pragma unroll
+  for (int m = 0; m < M; ++m) {
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      float g;
+      if (VAR == VAR_STANDARD) {
+        g = mean[e];                      // Alg. 1 line 10
+      } else if (VAR == VAR_DELAYED) {
+        g = pa[e];                        // Alg. 2 line 11
+      } else {
+        float t = d[m][e] - pl[m][e];     // Alg. 3 line 11
+        t = t / a.fM;
+        g = t + pa[e];
+      }
+      nesterov(g, a.eta, a.mu, b[m][e], s[m][e]);
+    }
+    F32Vec<V>::store(a.mom + m * a.stride + i, b[m]);
+    F32Vec<V>::store(a.start + m * a.stride + i, s[m]);
+    store_theta<TK, V>(a, m * a.stride + i, s[m]);
+    if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + m * a.stride + i, d[m]);
+  }
+  if (VAR != VAR_STANDARD) F32Vec<V>::store(a.dpa + i, mean);
+  }
+}
+
+// ---------------------------------------------------------------- outer step, runtime M
+// Two sweeps over the replicas: the first forms the mean, the second re-reads s_m and
+// theta_m (L1/L2 hits: the same thread read them a few hundred cycles earlier) and updates.
+template <int VAR, int TK, bool BOOT, int V>
+__device__ __forceinline__ void outer_column_rt(const OuterArgs &a, long long i) {
+  float mean[V];
+  for (int m = 0; m < a.M; ++m) {
+    float s[V], x[V];
+    F32Vec<V>::load_cached(a.start + m * a.stride + i, s);
+    load_theta<TK, V>(a, m * a.stride + i, x, true);
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      float dm = s[e] - x[e];
+      mean[e] = (m == 0) ? dm : mean[e] + dm;
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
+  float pa[V];
+  if (!BOOT && VAR != VAR_STANDARD) F32Vec<V>::load(a.dpa + i, pa);
+  for (int m = 0; m < a.M; ++m) {
+    float s[V], x[V], d[V];
+    F32Vec<V>::load_cached(a.start + m * a.stride + i, s);
+    load_theta<TK, V>(a, m * a.stride + i, x, true);
+#pragma unroll
+    for (int e = 0; e < V; ++e) d[e] = s[e] - x[e];
+    if (BOOT) {
+      F32Vec<V>::store(a.start + m * a.stride + i, x);
+      if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + m * a.stride + i, d);
+      continue;
+    }
+    float b[V], pl[V];
+    F32Vec<V>::load(a.mom + m * a.stride + i, b);
+    if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + m * a.stride + i, pl);
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      float g;
+      if (VAR == VAR_STANDARD) {
+        g = mean[e];
+      } else if (VAR == VAR_DELAYED) {
+        g = pa[e];
+      } else {
+        float t = d[e] - pl[e];
+        t = t / a.fM;
+        g = t + pa[e];
+      }
+      nesterov(g, a.eta, a.mu, b[e], s[e]);
+    }
+    F32Vec<V>::store(a.mom + m * a.stride + i, b);
+    F32Vec<V>::store(a.start + m * a.stride + i, s);
+    store_theta<TK, V>(a, m * a.stride + i, s);
+    if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + m * a.stride + i, d);
+  }
+  if (VAR != VAR_STANDARD) F32Vec<V>::store(a.dpa + i, mean);
+}
+
+// M = 0 selects the runtime-M form.
+template <int M, int VAR, int TK, bool BOOT, int V>
+__device__ __forceinline__ void outer_any_column(const OuterArgs &a, long long i) {
+  if (M > 0) outer_column<(M > 0 ? M : 1), VAR, TK, BOOT, V>(a, i);
+  else outer_column_rt<VAR, TK, BOOT, V>(a, i);
+}
+
+template <int M, int VAR, int TK, bool BOOT, int V, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) outer_step_kernel(const OuterArgs a) {
+  const long long nvec = a.P / V;
+  const long long nthreads = (long long)gridDim.x * kThreads;
+  const long long tid = (long long)blockIdx.x * kThreads + threadIdx.x;
+  for (long long j = tid; j < nvec; j += nthreads) outer_any_column<M, VAR, TK, BOOT, V>(a, j * V);
+  // ragged tail: P % V single indices
+  for (long long i = nvec * V + tid; i < a.P; i += nthreads) outer_any_column<M, VAR, TK, BOOT, 1>(a, i);
+}
+
+// ---------------------------------------------------------------- inner AdamW
+// U columns of one thread: all loads of all U columns are issued before the first use, so a
+// thread keeps U x (theta, g, m, v) vectors in flight.
+template <int TK, int GK, int V, int U>
+__device__ __forceinline__ void adamw_columns(const AdamArgs &a, int m, const long long (&idx)[U]) {
+  float g[U][V], x[U][V], m1[U][V], v1[U][V];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const long long at = m * a.stride + idx[u];
+    const long long gat = m * a.gstride + idx[u];
+    if (GK == GK_F32) F32Vec<V>::load(reinterpret_cast<const float *>(a.grads) + gat, g[u]);
+    else BF16Vec<V>::load(reinterpret_cast<const unsigned short *>(a.grads) + gat, g[u]);
+    if (TK == TK_F32) F32Vec<V>::load(reinterpret_cast<const float *>(a.theta) + at, x[u]);
+    else if (TK == TK_BF16) BF16Vec<V>::load(reinterpret_cast<const unsigned short *>(a.theta) + at, x[u]);
+    else F32Vec<V>::load(a.master + at, x[u]);
+    F32Vec<V>::load(a.m + at, m1[u]);
+    F32Vec<V>::load(a.v + at, v1[u]);
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      float t1 = a.beta1 * m1[u][e];
+      float t2 = a.omb1 * g[u][e];
+      m1[u][e] = t1 + t2;
+      float t3 = a.beta2 * v1[u][e];
+      float t4 = a.omb2 * g[u][e];
+      t4 = t4 * g[u][e];
+      v1[u][e] = t3 + t4;
+      float mh = m1[u][e] / a.c1;
+      float vh = v1[u][e] / a.c2;
+      float den = sqrtf(vh) + a.eps;
+      float r = mh / den;
+      float w = a.wd * x[u][e];
+      float upd = r + w;
+      upd = a.lr * upd;
+      x[u][e] = x[u][e] - upd;
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const long long at = m * a.stride + idx[u];
+    F32Vec<V>::store(a.m + at, m1[u]);
+    F32Vec<V>::store(a.v + at, v1[u]);
+    if (TK == TK_F32) {
+      F32Vec<V>::store(reinterpret_cast<float *>(a.theta) + at, x[u]);
+    } else if (TK == TK_BF16) {
+      BF16Vec<V>::store(reinterpret_cast<unsigned short *>(a.theta) + at, x[u]);
+    } else {
+      F32Vec<V>::store(a.master + at, x[u]);
+      BF16Vec<V>::store(reinterpret_cast<unsigned short *>(a.theta) + at, x[u]);
+    }
+  }
+}
+
+// grid = (blocks per replica, M)
+template <int TK, int GK, int V, int U>
+__global__ void __launch_bounds__(kThreads) adamw_kernel(const AdamArgs a) {
+  const int m = blockIdx.y;
+  const long long nvec = a.P / V;
+  const long long nthreads = (long long)gridDim.x * kThreads;
+  const long long tid = (long long)blockIdx.x * kThreads + threadIdx.x;
+  long long j = tid;
+  for (; j + (U - 1) * nthreads < nvec; j += U * nthreads) {
+    long long idx[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) idx[u] = (j + u * nthreads) * V;
+    adamw_columns<TK, GK, V, U>(a, m, idx);
+  }
+  for (; j < nvec; j += nthreads) {
+    long long idx[1] = {j * V};
+    adamw_columns<TK, GK, V, 1>(a, m, idx);
+  }
+  for (long long i = nvec * V + tid; i < a.P; i += nthreads) {
+    long long idx[1] = {i};
+    adamw_columns<TK, GK, 1, 1>(a, m, idx);
+  }
+}
+
+} // namespace diloco

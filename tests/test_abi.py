@@ -1,0 +1,124 @@
+"""Host-side checks that need no GPU: the shared library loads, exports every symbol the
+header declares, and rejects bad arguments with the documented status codes before touching
+the device."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+from paper_2502_12996_b200 import binding, build
+
+ROOT = Path(__file__).resolve().parent.parent
+HEADER = ROOT / "include" / "diloco.h"
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return binding.load_library()
+
+
+def declared_functions():
+    text = re.sub(r"/\*.*?\*/", "", HEADER.read_text(), flags=re.S)
+    return sorted(set(re.findall(r"\b(diloco_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/diloco.h but not exported"
+    assert sorted(binding.SYMBOLS) == names, "python binding and header disagree"
+
+
+def test_status_strings(lib):
+    seen = {binding.status_string(s) for s in range(0, -7, -1)}
+    assert len(seen) == 7 and "unknown status" not in seen
+    assert binding.status_string(-99) == "unknown status"
+    assert binding.launch_count() >= 0
+
+
+def good_config(**kw):
+    c = dict(M=4, H=30, P=1000, stride=1024, outer_lr=0.7, outer_momentum=0.9, beta1=0.9, beta2=0.95, eps=1e-8,
+             weight_decay=0.1, theta_kind=0, grad_kind=0, have_prev=1, impl=0)
+    c.update(kw)
+    return binding.Config(**c)
+
+
+def good_buffers(**kw):
+    b = {k: 0x10000 * (i + 1) for i, k in enumerate(
+        ["theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom", "adam_m", "adam_v"])}
+    b["device_status"] = None
+    b.update(kw)
+    return binding.Buffers(**b)
+
+
+def init(lib, cfg, buf):
+    h = ctypes.c_void_p()
+    rc = lib.diloco_state_init(ctypes.byref(cfg) if cfg is not None else None,
+                               ctypes.byref(buf) if buf is not None else None, ctypes.byref(h))
+    assert (rc == 0) == bool(h)
+    if h:
+        lib.diloco_state_free(h)
+    return rc
+
+
+@pytest.mark.parametrize("kw", [dict(M=0), dict(M=-3), dict(P=0), dict(stride=999), dict(theta_kind=3), dict(grad_kind=2),
+                                dict(outer_momentum=1.0), dict(outer_momentum=-0.1), dict(beta1=1.0), dict(beta2=-1.0),
+                                dict(eps=-1e-8), dict(weight_decay=-1.0), dict(have_prev=2), dict(impl=9),
+                                dict(outer_lr=float("nan")), dict(H=-1)])
+def test_invalid_config(lib, kw):
+    assert init(lib, good_config(**kw), good_buffers()) == binding.ERR_INVALID_ARG
+
+
+def test_unsupported_and_misaligned(lib):
+    assert init(lib, good_config(M=65), good_buffers()) == binding.ERR_UNSUPPORTED
+    assert init(lib, good_config(stride=1000 + 8), good_buffers()) == binding.ERR_MISALIGNED   # 4032 B rows
+    assert init(lib, good_config(stride=1024 + 32, theta_kind=1), good_buffers()) == binding.ERR_MISALIGNED  # bf16 rows
+    assert init(lib, good_config(), good_buffers(start=0x10008)) == binding.ERR_MISALIGNED
+    assert init(lib, good_config(), good_buffers(device_status=0x10002)) == binding.ERR_MISALIGNED
+
+
+def test_null_arguments(lib):
+    assert init(lib, None, good_buffers()) == binding.ERR_INVALID_ARG
+    assert init(lib, good_config(), None) == binding.ERR_INVALID_ARG
+    assert lib.diloco_state_init(ctypes.byref(good_config()), ctypes.byref(good_buffers()), None) == binding.ERR_INVALID_ARG
+    for missing in ("theta", "start", "outer_mom"):
+        assert init(lib, good_config(), good_buffers(**{missing: None})) == binding.ERR_INVALID_ARG
+    assert init(lib, good_config(theta_kind=2), good_buffers(master=None)) == binding.ERR_INVALID_ARG
+    assert init(lib, good_config(), good_buffers(adam_m=None)) == binding.ERR_INVALID_ARG      # moments come in pairs
+    assert lib.diloco_state_free(None) == 0
+    for fn in (lib.diloco_outer_eager, lib.diloco_outer_delayed, lib.diloco_outer_standard):
+        assert fn(None, None) == binding.ERR_INVALID_ARG
+    assert lib.diloco_inner_adamw(None, None, 0, 0.0, None) == binding.ERR_INVALID_ARG
+    assert lib.diloco_outer_fragment(None, 2, 0, 0, 1, None) == binding.ERR_INVALID_ARG
+    assert lib.diloco_state_set_counters(None, 0, 0, 0) == binding.ERR_INVALID_ARG
+    assert lib.diloco_set_outer_hparams(None, 0.1, 0.1) == binding.ERR_INVALID_ARG
+    assert lib.diloco_check_device_status(None, None) == binding.ERR_INVALID_ARG
+
+
+def test_valid_arguments_reach_the_device_query(lib):
+    """With valid arguments the only thing left is the device query: OK on a GPU machine, a CUDA
+    error (never a crash, never a silent CPU path) on a box without one."""
+    import torch
+    rc = init(lib, good_config(), good_buffers())
+    if torch.cuda.is_available():
+        assert rc == 0
+    else:
+        assert rc == binding.ERR_CUDA and binding.last_cuda_error() != 0
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", tmp_path / "libdiloco.so")
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.load_library()
+
+
+def test_product_does_not_import_the_oracle():
+    """The package may mention the checker in prose but must never import, load or include it."""
+    pkg = ROOT / "paper_2502_12996_b200"
+    pat = re.compile(r"^\s*(import\s+oracle|from\s+oracle|from\s+\.+\s*oracle)|libdiloco_oracle|oracle/|#include.*oracle", re.M)
+    for f in list(pkg.rglob("*.py")) + list(pkg.rglob("*.cu")) + list(pkg.rglob("*.cuh")):
+        assert not pat.search(f.read_text()), f

@@ -1,0 +1,286 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Bar: bit-exact for every fp32 buffer (both sides perform the same IEEE operations in the
+same order; FMA contraction is off on both), identical bit patterns for bf16 storage
+(tolerance 1 bf16 ulp allowed by the contract, 0 expected and asserted).  +0 and -0 compare
+equal.  All inputs are seeded and synthetic; the oracle receives copies of the device
+tensors, never a second draw.
+"""
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_12996_b200 import binding, inputs
+from gpu_util import (assert_state_equal, host_copy, oracle_adamw, oracle_outer, to_numpy, with_guards)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+HP = dict(lr=4e-4, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.1)
+NAMES = {0: "standard", 1: "delayed", 2: "eager"}
+
+
+def make(M, P, seed, theta_kind=0, with_adam=False, guards=True):
+    st = inputs.make_outer_state(M, P, seed, device=DEV, theta_kind=theta_kind, with_adam=with_adam)
+    # non-zero momentum and sentinel padding so that a wrong index or a write past P shows
+    st["outer_mom"][:, :P].normal_(0.0, 1e-3, generator=st["gen"])
+    for k in ("theta", "master", "start", "delta_prev_local", "outer_mom", "adam_m", "adam_v"):
+        if st.get(k) is not None:
+            st[k][:, P:] = 3.0
+    st["delta_prev_avg"][P:] = 3.0
+    checks = with_guards(st, DEV) if guards else []
+    return st, checks
+
+
+def run_outer_steps(oracle, variant, M, P, theta_kind, steps, seed, have_prev=1, eta=0.7, mu=0.9, impl=0):
+    st, checks = make(M, P, seed, theta_kind)
+    h = host_copy(st)
+    state = binding.State.from_dict(st, outer_lr=eta, outer_momentum=mu, have_prev=have_prev, impl=impl)
+    hp = have_prev
+    for k in range(steps):
+        if k > 0:
+            inputs.inner_phase_standin(st)
+            h["theta"] = to_numpy(st["theta"])
+            h["master"] = to_numpy(st["master"])
+        state.outer(variant)
+        oracle_outer(oracle, variant, h, M, P, st["stride"], eta, mu, theta_kind,
+                     bootstrap=(variant != 0 and hp == 0))
+        if variant != 0:
+            hp = 1
+        torch.cuda.synchronize()
+        assert_state_equal(st, h, what=f"{NAMES[variant]} M={M} P={P} kind={theta_kind} step {k + 1}")
+    for c in checks:
+        c()
+    assert state.get_counters()[1] == steps
+    state.close()
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("M,P", [(1, 70_001), (2, (1 << 20) + 3), (3, 100_003), (4, 300_007), (5, 50_001),
+                                 (8, 200_005), (16, 150_001), (64, 5_003)])
+def test_outer_fp32(oracle, variant, M, P):
+    run_outer_steps(oracle, variant, M, P, 0, steps=3, seed=100 + M)
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("theta_kind", [1, 2])
+@pytest.mark.parametrize("M,P", [(2, 100_001), (4, 250_003), (7, 20_001), (8, 60_002), (16, 40_003)])
+def test_outer_bf16_storage(oracle, variant, theta_kind, M, P):
+    run_outer_steps(oracle, variant, M, P, theta_kind, steps=3, seed=200 + M)
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("theta_kind", [0, 1, 2])
+@pytest.mark.parametrize("M", [2, 4, 6, 16])
+def test_first_outer_step_then_regular(oracle, variant, theta_kind, M):
+    """have_prev = 0: the first call records and applies nothing (t = H), later calls apply."""
+    run_outer_steps(oracle, variant, M, 33_335, theta_kind, steps=3, seed=300 + M, have_prev=0)
+
+
+@pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 63, 64, 65, 255, 1025])
+def test_tiny_and_ragged_sizes(oracle, P):
+    for variant in (0, 1, 2):
+        for M in (2, 4, 5):
+            run_outer_steps(oracle, variant, M, P, 0, steps=2, seed=400 + P)
+    run_outer_steps(oracle, 2, 4, P, 1, steps=2, seed=500 + P)
+    run_outer_steps(oracle, 2, 16, P, 2, steps=2, seed=600 + P)
+
+
+@pytest.mark.parametrize("eta,mu", [(0.4, 0.9), (1.0, 0.0), (0.7, 0.0)])
+def test_other_outer_hyperparameters(oracle, eta, mu):
+    run_outer_steps(oracle, 2, 4, 65_537, 0, steps=3, seed=700, eta=eta, mu=mu)
+    run_outer_steps(oracle, 0, 2, 65_537, 0, steps=2, seed=701, eta=eta, mu=mu)
+
+
+def test_worked_example_on_gpu():
+    """The hand-computed dyadic example (tests/golden): exact whatever the operation order."""
+    from test_oracle_outer import GOLDEN, VARIANTS, read_golden
+    g = read_golden(GOLDEN)
+    M, P, stride = 2, 2, 64
+    for name, variant in VARIANTS.items():
+        def dev(key, rows=M):
+            t = torch.zeros((rows, stride), dtype=torch.float32, device=DEV)
+            t[:, :P] = torch.tensor(g[key], dtype=torch.float32).view(rows, P)
+            return t
+        st = dict(theta=dev("theta"), start=dev("start"), delta_prev_local=dev("delta_prev_local"),
+                  delta_prev_avg=dev("delta_prev_avg", 1).view(-1), outer_mom=torch.zeros((M, stride), device=DEV))
+        state = binding.State(M=M, P=P, stride=stride, outer_lr=g["eta"][0], outer_momentum=g["mu"][0], **st)
+        for k in (1, 2):
+            if k == 2:
+                st["theta"][:, :P] += torch.tensor(g["inner_phase_2"], device=DEV).view(M, P)
+            state.outer(variant)
+            torch.cuda.synchronize()
+            want = torch.tensor(g[f"{name}_theta_{k}"]).view(M, P)
+            assert torch.equal(st["theta"][:, :P].cpu(), want), (name, k)
+            assert torch.equal(st["start"][:, :P].cpu(), want)
+            assert torch.equal(st["outer_mom"][:, :P].cpu(), torch.tensor(g[f"{name}_mom_{k}"]).view(M, P))
+        state.close()
+
+
+# ---------------------------------------------------------------- inner AdamW
+def run_adamw(oracle, M, P, theta_kind, grad_kind, steps, seed, segments=0):
+    st, checks = make(M, P, seed, theta_kind, with_adam=True)
+    stride = st["stride"]
+    h = host_copy(st)
+    state = binding.State.from_dict(st, grad_kind=grad_kind, beta1=HP["beta1"], beta2=HP["beta2"], eps=HP["eps"],
+                                    weight_decay=HP["wd"])
+    seg_sizes = seg_scales = None
+    if segments:
+        seg_sizes = inputs.segment_sizes(P, segments, d_model=16)
+        seg_scales = inputs.segment_scales(segments, st["gen"], DEV)
+    for k in range(1, steps + 1):
+        g = inputs.make_grads(M, P, stride, st["gen"], DEV, grad_kind, seg_sizes=seg_sizes, seg_scales=seg_scales)
+        state.inner_adamw(g, HP["lr"])
+        oracle_adamw(oracle, h, to_numpy(g), M, P, stride, stride, k, HP, theta_kind, grad_kind)
+        torch.cuda.synchronize()
+        assert_state_equal(st, h, what=f"adamw M={M} P={P} kind={theta_kind}/{grad_kind} step {k}")
+    for c in checks:
+        c()
+    assert state.get_counters()[0] == steps
+    state.close()
+    return st, h
+
+
+@pytest.mark.parametrize("theta_kind,grad_kind", [(0, 0), (0, 1), (1, 0), (1, 1), (2, 0), (2, 1)])
+@pytest.mark.parametrize("M,P", [(1, 10_001), (2, 1_000_003), (4, 300_005), (5, 777)])
+def test_adamw(oracle, theta_kind, grad_kind, M, P):
+    run_adamw(oracle, M, P, theta_kind, grad_kind, steps=4, seed=800 + M)
+
+
+def test_adamw_segment_scaled_gradients(oracle):
+    """Gradients with per-segment scales spread over two decades (the fourth configuration's law)."""
+    run_adamw(oracle, 4, 200_003, 2, 1, steps=3, seed=900, segments=256)
+
+
+@pytest.mark.parametrize("P", [1, 3, 4, 7, 64, 2049])
+def test_adamw_tiny(oracle, P):
+    run_adamw(oracle, 3, P, 0, 0, steps=2, seed=950 + P)
+    run_adamw(oracle, 2, P, 1, 1, steps=2, seed=960 + P)
+
+
+# ---------------------------------------------------------------- whole simulated phases
+@pytest.mark.parametrize("theta_kind,grad_kind", [(0, 0), (1, 1), (2, 1)])
+def test_full_phases(oracle, theta_kind, grad_kind):
+    """H inner AdamW steps on every replica, then one eager outer step; 3 phases, the first
+    outer step being the t = H bootstrap."""
+    M, P, H, phases = 4, 120_007, 5, 3
+    st, checks = make(M, P, 1000 + theta_kind, theta_kind, with_adam=True)
+    st["outer_mom"].zero_()
+    stride = st["stride"]
+    h = host_copy(st)
+    state = binding.State.from_dict(st, H=H, grad_kind=grad_kind, have_prev=0, beta1=HP["beta1"], beta2=HP["beta2"],
+                                    eps=HP["eps"], weight_decay=HP["wd"])
+    k = 0
+    for ph in range(phases):
+        for _ in range(H):
+            k += 1
+            g = inputs.make_grads(M, P, stride, st["gen"], DEV, grad_kind)
+            state.inner_adamw(g, HP["lr"])
+            oracle_adamw(oracle, h, to_numpy(g), M, P, stride, stride, k, HP, theta_kind, grad_kind)
+        state.outer_eager()
+        oracle_outer(oracle, 2, h, M, P, stride, 0.7, 0.9, theta_kind, bootstrap=(ph == 0))
+        torch.cuda.synchronize()
+        assert_state_equal(st, h, what=f"phase {ph + 1} kind={theta_kind}")
+    assert state.get_counters() == (H * phases, phases, 1)
+    for c in checks:
+        c()
+
+
+# ---------------------------------------------------------------- fragments, resume, host path
+@pytest.mark.parametrize("theta_kind", [0, 1])
+def test_fragments_equal_whole(oracle, theta_kind):
+    """Every index is independent: the step applied fragment by fragment (as a streaming
+    schedule would) gives the same bits as one call over the whole vector."""
+    M, P = 4, 200_003
+    a, _ = make(M, P, 1100, theta_kind)
+    b = {k: (v.clone() if torch.is_tensor(v) else v) for k, v in a.items()}
+    sa = binding.State.from_dict(a)
+    sb = binding.State.from_dict(b)
+    sa.outer_eager()
+    cuts = [0, 64 * 100, 64 * 1000, 64 * 1001, 64 * 3000, P]
+    for lo, hi in reversed(list(zip(cuts[:-1], cuts[1:]))):
+        sb.outer_fragment(binding.EAGER, False, lo, hi - lo)
+    torch.cuda.synchronize()
+    for k in ("theta", "start", "delta_prev_local", "delta_prev_avg", "outer_mom"):
+        assert torch.equal(a[k].view(torch.int16 if a[k].dtype == torch.bfloat16 else torch.int32),
+                           b[k].view(torch.int16 if b[k].dtype == torch.bfloat16 else torch.int32)), k
+    with pytest.raises(binding.DilocoError) as e:
+        sb.outer_fragment(binding.EAGER, False, 32 if theta_kind else 16, 100)
+    assert e.value.status == binding.ERR_MISALIGNED
+    with pytest.raises(binding.DilocoError) as e:
+        sb.outer_fragment(binding.EAGER, False, 64, P)
+    assert e.value.status == binding.ERR_INVALID_ARG
+
+
+def test_resume_from_counters(oracle):
+    """3 steps in one state == 1 step, state dropped, new state with restored counters, 2 steps."""
+    M, P = 2, 50_001
+    a, _ = make(M, P, 1200, 0, with_adam=True)
+    b = {k: (v.clone() if torch.is_tensor(v) else v) for k, v in a.items()}
+    gs = [inputs.make_grads(M, P, a["stride"], a["gen"], DEV, 0) for _ in range(3)]
+    sa = binding.State.from_dict(a, have_prev=0)
+    for g in gs:
+        sa.inner_adamw(g, 1e-3)
+        sa.outer_eager()
+    sb = binding.State.from_dict(b, have_prev=0)
+    sb.inner_adamw(gs[0], 1e-3)
+    sb.outer_eager()
+    counters = sb.get_counters()
+    sb.close()
+    sc = binding.State.from_dict(b, have_prev=0)
+    sc.set_counters(*counters)
+    for g in gs[1:]:
+        sc.inner_adamw(g, 1e-3)
+        sc.outer_eager()
+    torch.cuda.synchronize()
+    for k in ("theta", "start", "delta_prev_local", "delta_prev_avg", "outer_mom", "adam_m", "adam_v"):
+        assert torch.equal(a[k], b[k]), k
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("theta_kind", [0, 2])
+def test_host_buffer_entry_point(oracle, variant, theta_kind):
+    """State in pinned host memory, chunked copy-in / step / copy-out: same bits as the oracle."""
+    M, P = 4, 300_001
+    st, _ = make(M, P, 1300 + variant, theta_kind, guards=False)
+    h = host_copy(st)
+    pinned = {k: (st[k].cpu().pin_memory() if st.get(k) is not None else None)
+              for k in ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom")}
+    for k in ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom"):
+        if st.get(k) is not None:
+            st[k].fill_(-7.0)                                     # the device copy must come from the host
+    state = binding.State.from_dict(st)
+    streams = [torch.cuda.Stream(device=DEV) for _ in range(3)]
+    host = binding.make_buffers(**pinned)
+    for step in range(2):
+        state.outer_step_host(variant, host, streams, 64 * 1000)
+        streams[2].synchronize()
+        oracle_outer(oracle, variant, h, M, P, st["stride"], 0.7, 0.9, theta_kind)
+        assert_state_equal(pinned, h, keys=tuple(pinned), what=f"host path {NAMES[variant]} step {step + 1}")
+    state.close()
+
+
+def test_launch_counter():
+    M, P = 2, 1000
+    st, _ = make(M, P, 1400, 0, with_adam=True)
+    state = binding.State.from_dict(st)
+    n0 = binding.launch_count()
+    state.outer_eager()
+    state.outer_standard()
+    state.inner_adamw(torch.zeros((M, st["stride"]), device=DEV), 1e-3)
+    assert binding.launch_count() == n0 + 3
+    torch.cuda.synchronize()
+
+
+def test_non_default_stream(oracle):
+    M, P = 4, 100_001
+    st, _ = make(M, P, 1500, 0)
+    h = host_copy(st)
+    state = binding.State.from_dict(st)
+    s = torch.cuda.Stream(device=DEV)
+    s.wait_stream(torch.cuda.current_stream())
+    state.outer_eager(stream=s)
+    s.synchronize()
+    oracle_outer(oracle, 2, h, M, P, st["stride"], 0.7, 0.9, 0)
+    assert_state_equal(st, h)
