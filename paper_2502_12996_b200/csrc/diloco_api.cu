@@ -11,6 +11,7 @@
 #include <new>
 #include <vector>
 
+#include "diloco_bulk.cuh"
 #include "diloco_kernels.cuh"
 
 using namespace diloco;
@@ -72,39 +73,27 @@ int validate_buffers(const diloco_config_t *c, const diloco_buffers_t *b) {
   return DILOCO_OK;
 }
 
-// blocks to launch for `work` columns: a persistent grid of (resident blocks per SM) x SMs
-template <typename K>
-int grid_for(K kernel, const diloco_state *st, long long work, int *grid) {
-  int per_sm = 0;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0);
-  if (e != cudaSuccess) return cuda_fail(e);
-  if (per_sm < 1) per_sm = 1;
-  long long need = (work + kThreads - 1) / kThreads;
-  long long cap = (long long)per_sm * st->sm_count;
-  if (need < 1) need = 1;
-  *grid = (int)(need < cap ? need : cap);
-  return DILOCO_OK;
-}
-
-template <int M, int VAR, int TK, bool BOOT, int V, int MINB>
-int launch_outer_t(const diloco_state *st, const OuterArgs &a, cudaStream_t s) {
-  auto k = outer_step_kernel<M, VAR, TK, BOOT, V, MINB>;
-  int grid = 1;
-  int rc = grid_for(k, st, (a.P + V - 1) / V, &grid);
-  if (rc != DILOCO_OK) return rc;
-  k<<<grid, kThreads, 0, s>>>(a);
+template <int M, int G, int VAR, int TK, bool BOOT, int V, int NT, int MINB>
+int launch_outer_t(const OuterArgs &a, cudaStream_t s) {
+  constexpr int CW = 32 / G;
+  const long long nvec = a.P / V;
+  const long long warps = (nvec + CW - 1) / CW;
+  long long blocks = (warps * 32 + NT - 1) / NT;
+  if (blocks < 1) blocks = 1; // the last block also handles the P % V tail
+  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
+  outer_step_kernel<M, G, VAR, TK, BOOT, V, NT, MINB><<<(unsigned)blocks, NT, 0, s>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1);
   return DILOCO_OK;
 }
 
-template <int M, int V, int MINB>
-int launch_outer_m(const diloco_state *st, int var, int tk, bool boot, const OuterArgs &a, cudaStream_t s) {
-#define DILOCO_CASE(VAR_, TK_)                                                            \
-  if (var == VAR_ && tk == TK_) {                                                         \
-    if (VAR_ != VAR_STANDARD && boot) return launch_outer_t<M, VAR_, TK_, true, V, MINB>(st, a, s); \
-    return launch_outer_t<M, VAR_, TK_, false, V, MINB>(st, a, s);                         \
+template <int M, int G, int V, int NT, int MINB>
+int launch_outer_m(int var, int tk, bool boot, const OuterArgs &a, cudaStream_t s) {
+#define DILOCO_CASE(VAR_, TK_)                                                                           \
+  if (var == VAR_ && tk == TK_) {                                                                        \
+    if (VAR_ != VAR_STANDARD && boot) return launch_outer_t<M, G, VAR_, TK_, true, V, NT, MINB>(a, s);   \
+    return launch_outer_t<M, G, VAR_, TK_, false, V, NT, MINB>(a, s);                                    \
   }
   DILOCO_CASE(VAR_STANDARD, TK_F32)
   DILOCO_CASE(VAR_STANDARD, TK_BF16)
@@ -119,16 +108,23 @@ int launch_outer_m(const diloco_state *st, int var, int tk, bool boot, const Out
   return DILOCO_ERR_INVALID_ARG;
 }
 
+// Launch shapes per M (lane groups G, vector width V, threads NT, min resident blocks MINB),
+// chosen by measurement on B200 under two rules: no register spills, and every warp-level
+// access covers at least 128 contiguous bytes of a row (64-byte runs halved the bandwidth).
+// M <= 3: one thread per column.  M = 4, 8, 16: the replica axis is split over G lanes.
 int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterArgs &a, cudaStream_t s) {
   const int tk = st->cfg.theta_kind;
   switch (st->cfg.M) {
-    case 1: return launch_outer_m<1, 4, 4>(st, var, tk, boot, a, s);
-    case 2: return launch_outer_m<2, 4, 3>(st, var, tk, boot, a, s);
-    case 3: return launch_outer_m<3, 4, 2>(st, var, tk, boot, a, s);
-    case 4: return launch_outer_m<4, 4, 2>(st, var, tk, boot, a, s);
-    case 8: return launch_outer_m<8, 4, 1>(st, var, tk, boot, a, s);
-    case 16: return launch_outer_m<16, 2, 1>(st, var, tk, boot, a, s);
-    default: return launch_outer_m<0, 4, 2>(st, var, tk, boot, a, s);
+    case 1: return launch_outer_m<1, 1, 4, 128, 8>(var, tk, boot, a, s);
+    case 2: return launch_outer_m<2, 1, 4, 128, 6>(var, tk, boot, a, s);
+    case 3: return launch_outer_m<3, 1, 4, 128, 4>(var, tk, boot, a, s);
+    case 4: return launch_outer_m<4, 2, 4, 128, 8>(var, tk, boot, a, s);
+    case 8:
+      // fp32 rows: 16 lanes x 8 B = 128 B per row; bf16 rows need the wider vector for that
+      if (tk == TK_F32) return launch_outer_m<8, 2, 2, 256, 3>(var, tk, boot, a, s);
+      return launch_outer_m<8, 2, 4, 128, 4>(var, tk, boot, a, s);
+    case 16: return launch_outer_m<16, 4, 4, 128, 4>(var, tk, boot, a, s);
+    default: return launch_outer_m<0, 1, 4, 128, 4>(var, tk, boot, a, s);
   }
 }
 
@@ -158,8 +154,54 @@ OuterArgs outer_args(const diloco_state *st, int64_t offset, int64_t len) {
   return a;
 }
 
+// Bulk (TMA-staged) form: one CTA ring per SM slot, grid capped by the tile count.
+template <int M, int VAR, int TK, int T, int S, int NT>
+int launch_bulk_t(const diloco_state *st, const OuterArgs &a, cudaStream_t s) {
+  auto k = outer_step_bulk_kernel<M, VAR, TK, T, S, NT>;
+  constexpr int smem = S * BulkStage<M, VAR, TK, T>::kBytes;
+  static_assert(smem <= 227 * 1024, "stage ring exceeds the shared memory of one SM");
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return cuda_fail(e);
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, NT, smem);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (per_sm < 1) per_sm = 1;
+  long long grid = (long long)per_sm * st->sm_count;
+  const long long ntiles = a.P / T;
+  if (grid > ntiles) grid = ntiles;
+  k<<<(unsigned)grid, NT, smem, s>>>(a, st->buf.device_status);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1);
+  return DILOCO_OK;
+}
+
+template <int M, int T, int S, int NT>
+int launch_bulk_m(const diloco_state *st, int var, int tk, const OuterArgs &a, cudaStream_t s) {
+#define DILOCO_CASE(VAR_, TK_) \
+  if (var == VAR_ && tk == TK_) return launch_bulk_t<M, VAR_, TK_, T, S, NT>(st, a, s);
+  DILOCO_CASE(VAR_STANDARD, TK_F32)
+  DILOCO_CASE(VAR_STANDARD, TK_BF16)
+  DILOCO_CASE(VAR_STANDARD, TK_MASTER_BF16)
+  DILOCO_CASE(VAR_DELAYED, TK_F32)
+  DILOCO_CASE(VAR_DELAYED, TK_BF16)
+  DILOCO_CASE(VAR_DELAYED, TK_MASTER_BF16)
+  DILOCO_CASE(VAR_EAGER, TK_F32)
+  DILOCO_CASE(VAR_EAGER, TK_BF16)
+  DILOCO_CASE(VAR_EAGER, TK_MASTER_BF16)
+#undef DILOCO_CASE
+  return DILOCO_ERR_INVALID_ARG;
+}
+
 int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t len, cudaStream_t s) {
   OuterArgs a = outer_args(st, offset, len);
+  // The bulk form exists for M = 2 and M = 4 only, needs the status word for its bounded
+  // waits and at least one full tile; everything else (and AUTO) takes the direct form,
+  // which measured faster at every M.
+  if (st->cfg.impl == DILOCO_IMPL_BULK && !boot && st->buf.device_status) {
+    if (st->cfg.M == 2 && len >= 1024) return launch_bulk_m<2, 1024, 3, 256>(st, var, st->cfg.theta_kind, a, s);
+    if (st->cfg.M == 4 && len >= 512) return launch_bulk_m<4, 512, 3, 128>(st, var, st->cfg.theta_kind, a, s);
+  }
   return launch_outer_direct(st, var, boot, a, s);
 }
 
@@ -177,20 +219,14 @@ int outer_whole(diloco_state *st, int var, void *stream) {
 
 template <int TK, int GK>
 int launch_adamw_t(const diloco_state *st, const AdamArgs &a, cudaStream_t s) {
-  constexpr int V = 4, U = 2;
-  auto k = adamw_kernel<TK, GK, V, U>;
-  int per_sm = 0;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, 0);
-  if (e != cudaSuccess) return cuda_fail(e);
-  if (per_sm < 1) per_sm = 1;
-  const int M = st->cfg.M;
-  long long need = ((a.P + V - 1) / V + (long long)kThreads * U - 1) / ((long long)kThreads * U);
-  long long cap = ((long long)per_sm * st->sm_count + M - 1) / M; // resident blocks shared by the M rows
-  if (need < 1) need = 1;
-  if (cap < 1) cap = 1;
-  dim3 grid((unsigned)(need < cap ? need : cap), (unsigned)M);
-  k<<<grid, kThreads, 0, s>>>(a);
-  e = cudaGetLastError();
+  constexpr int V = 4, U = 1, NT = 256, MINB = 4;
+  const long long nvec = a.P / V;
+  long long blocks = (nvec + (long long)NT * U - 1) / ((long long)NT * U);
+  if (blocks < 1) blocks = 1;
+  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
+  dim3 grid((unsigned)blocks, (unsigned)st->cfg.M);
+  adamw_kernel<TK, GK, V, U, NT, MINB><<<grid, NT, 0, s>>>(a);
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1);
   return DILOCO_OK;

@@ -36,7 +36,9 @@ def make(M, P, seed, theta_kind=0, with_adam=False, guards=True):
 def run_outer_steps(oracle, variant, M, P, theta_kind, steps, seed, have_prev=1, eta=0.7, mu=0.9, impl=0):
     st, checks = make(M, P, seed, theta_kind)
     h = host_copy(st)
-    state = binding.State.from_dict(st, outer_lr=eta, outer_momentum=mu, have_prev=have_prev, impl=impl)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    state = binding.State.from_dict(st, outer_lr=eta, outer_momentum=mu, have_prev=have_prev, impl=impl,
+                                    device_status=status)
     hp = have_prev
     for k in range(steps):
         if k > 0:
@@ -53,6 +55,8 @@ def run_outer_steps(oracle, variant, M, P, theta_kind, steps, seed, have_prev=1,
     for c in checks:
         c()
     assert state.get_counters()[1] == steps
+    state.check_device_status()
+    assert int(status.item()) == 0
     state.close()
 
 
@@ -85,6 +89,15 @@ def test_tiny_and_ragged_sizes(oracle, P):
             run_outer_steps(oracle, variant, M, P, 0, steps=2, seed=400 + P)
     run_outer_steps(oracle, 2, 4, P, 1, steps=2, seed=500 + P)
     run_outer_steps(oracle, 2, 16, P, 2, steps=2, seed=600 + P)
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("theta_kind", [0, 1, 2])
+@pytest.mark.parametrize("M,P", [(2, 700_003), (4, 400_005), (4, 511), (2, 1024)])
+def test_bulk_staged_implementation(oracle, variant, theta_kind, M, P):
+    """The TMA-staged form (tiles through shared memory, bounded mbarrier waits) must give the
+    same bits as the oracle, including the ragged tail and sizes below one tile."""
+    run_outer_steps(oracle, variant, M, P, theta_kind, steps=3, seed=650 + M, impl=binding.IMPL_BULK)
 
 
 @pytest.mark.parametrize("eta,mu", [(0.4, 0.9), (1.0, 0.0), (0.7, 0.0)])
