@@ -39,7 +39,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per parameter index for one launch of the
 # dominant kernel, from the captures summarised under profiles/ (None: not captured yet).
-NCU_TRAFFIC_BYTES_PER_PARAM = {}
+NCU_TRAFFIC_BYTES_PER_PARAM = {
+    ("diloco_outer_eager", 4, 0): 134.37,    # profiles/outer_eager_f32_M4_P35M_cfg1.md
+    ("diloco_inner_adamw", 4, 1): 86.34,     # profiles/inner_adamw_bf16_M4_P35M_cfg2slice.md (35 M slice, scaled by P)
+}
 
 
 def outer_bytes_per_param(variant: int, M: int, theta_kind: int) -> int:
