@@ -205,3 +205,15 @@ def make_grads(M: int, P: int, gstride: int, gen: torch.Generator, device, grad_
                 z *= seg_scales[seg]
             out[m, a:b].copy_(z)
     return out
+
+
+def make_segment_grads(M: int, seg_sizes: List[int], seg_scales: List[float], gen: torch.Generator,
+                       out: torch.Tensor) -> torch.Tensor:
+    """g_i = sigma_seg(i) * N(0, 1), drawn segment by segment straight into `out` [M, >= P]
+    (no full-size temporaries: for vectors that nearly fill the device)."""
+    for m in range(M):
+        lo = 0
+        for size, sigma in zip(seg_sizes, seg_scales):
+            out[m, lo:lo + size].normal_(0.0, float(sigma), generator=gen)
+            lo += size
+    return out

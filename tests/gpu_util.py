@@ -10,8 +10,8 @@ KEYS = ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer
 
 def to_numpy(t):
     """Device tensor -> host numpy array; bf16 as uint16 bit patterns."""
-    if t is None:
-        return None
+    if t is None or isinstance(t, np.ndarray):
+        return t
     t = t.detach().cpu()
     if t.dtype == torch.bfloat16:
         return t.contiguous().view(torch.int16).numpy().view(np.uint16).copy()
