@@ -226,7 +226,12 @@ def run_ours(args):
                                     impl=args.kernel)
     grads = None
     if phase:
-        grads = inputs.make_grads(M, P, stride, st["gen"], dev, w.grad_kind)
+        if w.segments:
+            grads = torch.zeros((M, stride), dtype=torch.bfloat16 if w.grad_kind else torch.float32, device=dev)
+            inputs.make_segment_grads(M, inputs.segment_sizes(P, w.segments),
+                                      inputs.segment_scales(w.segments, st["gen"], dev).tolist(), st["gen"], grads)
+        else:
+            grads = inputs.make_grads(M, P, stride, st["gen"], dev, w.grad_kind)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     outer_bpp = outer_bytes_per_param(variant, M, w.theta_kind)
     adam_bpp = adamw_bytes_per_param(M, w.theta_kind, w.grad_kind)
