@@ -25,6 +25,7 @@ _LIB = _HERE / "libdiloco_oracle.so"
 STANDARD, DELAYED, EAGER = 0, 1, 2
 THETA_NATIVE, THETA_BF16, THETA_MASTER_BF16 = 0, 1, 2
 GRAD_NATIVE, GRAD_BF16 = 0, 1
+COMM_F32, COMM_BF16, COMM_EXMY = 0, 1, 2
 
 _lib = None
 
@@ -75,7 +76,8 @@ def _theta_dtype(theta_kind, real):
 
 def outer_step(variant, *, M, P, stride, eta, mu, theta, start, outer_mom,
                delta_prev_local=None, delta_prev_avg=None, master=None,
-               theta_kind=THETA_NATIVE, bootstrap=False, nthreads=1):
+               theta_kind=THETA_NATIVE, bootstrap=False, nthreads=1,
+               comm=COMM_F32, exp_bits=0, man_bits=0, scales_out=None):
     """One outer step of Algorithm 1 (STANDARD), 2 (DELAYED) or 3 (EAGER), in place.
 
     ``theta`` is float32/float64 [M, stride] for THETA_NATIVE, else uint16 bf16 bit patterns;
@@ -89,14 +91,15 @@ def outer_step(variant, *, M, P, stride, eta, mu, theta, start, outer_mom,
         raise ValueError("delayed/eager need delta_prev_avg")
     if theta_kind == THETA_MASTER_BF16 and master is None:
         raise ValueError("master copy missing")
-    fn = getattr(lib(), f"oracle_outer_step_{sfx}")
+    fn = getattr(lib(), f"oracle_outer_step_comm_{sfx}")
     fn.restype = ctypes.c_int
     fn.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
-                   creal, creal, ctypes.c_int] + [ctypes.c_void_p] * 6 + [ctypes.c_int]
+                   creal, creal, ctypes.c_int] + [ctypes.c_void_p] * 6 \
+                  + [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_int]
     rc = fn(variant, int(bool(bootstrap)), M, P, stride, eta, mu, theta_kind,
             _ptr(theta, _theta_dtype(theta_kind, real)), _ptr(master, real), _ptr(start, real),
             _ptr(delta_prev_local, real), _ptr(delta_prev_avg, real), _ptr(outer_mom, real),
-            int(nthreads))
+            int(comm), int(exp_bits), int(man_bits), _ptr(scales_out, real), int(nthreads))
     if rc != 0:
         raise ValueError("oracle_outer_step rejected its arguments")
 
@@ -141,6 +144,21 @@ def inner_adamw(*, M, P, stride, gstride, lr, beta1, beta2, eps, wd, k, theta, g
             _ptr(adam_m, real), _ptr(adam_v, real), int(nthreads))
     if rc != 0:
         raise ValueError("oracle_inner_adamw rejected its arguments")
+
+
+def exmy_round(y: float, exp_bits: int, man_bits: int) -> float:
+    """Nearest EXMY(exp_bits, man_bits) number (ties to the even code, saturating)."""
+    fn = lib().oracle_exmy_round_f64
+    fn.restype = ctypes.c_double
+    fn.argtypes = [ctypes.c_double, ctypes.c_int, ctypes.c_int]
+    return float(fn(y, exp_bits, man_bits))
+
+
+def exmy_max(exp_bits: int, man_bits: int) -> float:
+    fn = lib().oracle_exmy_max_f64
+    fn.restype = ctypes.c_double
+    fn.argtypes = [ctypes.c_int, ctypes.c_int]
+    return float(fn(exp_bits, man_bits))
 
 
 def f32_to_bf16(x: float) -> int:

@@ -28,6 +28,16 @@
  *   - 1/M is a division by (REAL)M; the sum over m runs left to right.
  *   - InnerOpt = AdamW with decoupled weight decay, bias correction,
  *     eps added after the square root.
+ *   - Quantised communication (Section 3, "Quantized Communication": outer
+ *     gradients sent as float32, bfloat16, float8 or float4 "using EXMY"): the
+ *     operand of the all-reduce, and only it, is rounded: Delta = (1/M) sum_m
+ *     Q_m(Delta_m); every local use of Delta_m (line 11's fresh and stale
+ *     terms) stays in full precision.  The paper fixes no bit layout, so EXMY
+ *     is read as: 1 sign bit, X exponent bits, Y mantissa bits, bias
+ *     2^(X-1)-1, subnormals, every code a finite number (no inf/NaN codes),
+ *     round to nearest with ties to the even code, saturating; each replica's
+ *     vector is scaled so that its largest magnitude maps to the format's
+ *     largest value (one fp32 scale per replica per outer step).
  *
  * Parity pins: every function here is pinned by tests/test_oracle_*.py
  * (hand-worked dyadic example, exact rational brute force, closed forms,
@@ -94,6 +104,69 @@ static void store_theta(int kind, void *theta, REAL *master, size_t at, REAL x)
     }
 }
 
+/* communication format of the outer gradients */
+enum { COMM_F32 = 0, COMM_BF16 = 1, COMM_EXMY = 2 };
+
+/* largest finite EXMY value: top exponent code, all mantissa bits set */
+static double exmy_max(int X, int Y)
+{
+    int bias = (1 << (X - 1)) - 1;
+    int emax = (1 << X) - 1 - bias;
+    return ldexp(2.0 - ldexp(1.0, -Y), emax);
+}
+
+/* the (X+Y)-bit code of a non-negative representable value v: exponent field << Y | mantissa */
+static int exmy_code(double v, int X, int Y)
+{
+    int bias = (1 << (X - 1)) - 1;
+    if (v < ldexp(1.0, 1 - bias)) return (int)(v / ldexp(1.0, 1 - bias - Y));   /* subnormal: field 0 */
+    int e2;
+    double f = frexp(v, &e2);           /* v = f * 2^e2, 0.5 <= f < 1 */
+    int E = e2 - 1;
+    int mant = (int)((2.0 * f - 1.0) * (double)(1 << Y));
+    (void)X;
+    return ((E + bias) << Y) | mant;
+}
+
+/*
+ * Nearest EXMY(X, Y) number to y, ties to the even code, saturating.  Within
+ * the binade 2^E <= |y| < 2^(E+1) the representable numbers are the multiples
+ * of 2^(E-Y); below the smallest normal 2^(1-bias) the spacing stays
+ * 2^(1-bias-Y) (subnormals).  The two neighbours are lo = floor(|y|/spacing) *
+ * spacing and hi = lo + spacing (2^(E+1) when lo is the binade's last number);
+ * all of this is exact in double.
+ */
+static double exmy_round(double y, int X, int Y)
+{
+    double a = fabs(y);
+    if (a == 0.0 || a != a) return y;
+    int bias = (1 << (X - 1)) - 1;
+    int e2;
+    (void)frexp(a, &e2);               /* a = f * 2^e2, 0.5 <= f < 1  =>  2^(e2-1) <= a */
+    int E = e2 - 1;
+    if (E < 1 - bias) E = 1 - bias;
+    double spacing = ldexp(1.0, E - Y);
+    double lo = floor(a / spacing) * spacing;
+    double hi = lo + spacing;
+    double q;
+    if (a - lo < hi - a) q = lo;
+    else if (a - lo > hi - a) q = hi;
+    else q = (exmy_code(lo, X, Y) % 2 == 0) ? lo : hi;
+    double top = exmy_max(X, Y);
+    if (q > top) q = top;
+    return y < 0 ? -q : q;
+}
+
+/* what the wire carries for one element of replica m's outer gradient */
+static REAL comm_round(REAL d, int comm, int X, int Y, REAL scale)
+{
+    if (comm == COMM_F32) return d;
+    if (comm == COMM_BF16) return (REAL)bf16_to_f32(f32_to_bf16_rne((float)d));
+    REAL y = d / scale;
+    REAL q = (REAL)exmy_round((double)y, X, Y);
+    return q * scale;
+}
+
 /*
  * One outer step at index range [0, P) for all M replicas.
  *
@@ -110,16 +183,34 @@ static void store_theta(int kind, void *theta, REAL *master, size_t at, REAL x)
  * (eager only), delta_prev_avg [stride] (delayed, eager), outer_mom
  * [M,stride].  All updated in place.  Returns 0, or -1 on a bad argument.
  */
-int FN(oracle_outer_step)(int variant, int bootstrap, int M, int64_t P, int64_t stride,
-                          REAL eta, REAL mu, int theta_kind,
-                          void *theta, REAL *master, REAL *start,
-                          REAL *delta_prev_local, REAL *delta_prev_avg, REAL *outer_mom,
-                          int nthreads)
+int FN(oracle_outer_step_comm)(int variant, int bootstrap, int M, int64_t P, int64_t stride,
+                               REAL eta, REAL mu, int theta_kind,
+                               void *theta, REAL *master, REAL *start,
+                               REAL *delta_prev_local, REAL *delta_prev_avg, REAL *outer_mom,
+                               int comm, int X, int Y, REAL *scales_out, int nthreads)
 {
     if (M < 1 || M > 64 || P < 0 || stride < P) return -1;
     if (variant < VAR_STANDARD || variant > VAR_EAGER) return -1;
     if (variant == VAR_STANDARD && bootstrap) return -1;
+    if (comm < COMM_F32 || comm > COMM_EXMY) return -1;
+    if (comm == COMM_EXMY && (X < 1 || X > 5 || Y < 0 || X + Y > 7)) return -1;
     (void)nthreads;
+    /* per-replica scale: largest |Delta_m| maps to the largest EXMY value */
+    REAL scale[64];
+    for (int m = 0; m < M; ++m) scale[m] = (REAL)1;
+    if (comm == COMM_EXMY) {
+        for (int m = 0; m < M; ++m) {
+            REAL amax = (REAL)0;
+            for (int64_t i = 0; i < P; ++i) {
+                size_t at = (size_t)m * (size_t)stride + (size_t)i;
+                REAL dm = start[at] - load_theta(theta_kind, theta, master, at);
+                REAL ab = dm < 0 ? -dm : dm;
+                if (ab > amax) amax = ab;
+            }
+            if (amax > (REAL)0) scale[m] = amax / (REAL)exmy_max(X, Y);
+            if (scales_out) scales_out[m] = scale[m];
+        }
+    }
 #pragma omp parallel for schedule(static) num_threads(nthreads > 0 ? nthreads : 1)
     for (int64_t i = 0; i < P; ++i) {
         REAL d[64];
@@ -129,9 +220,10 @@ int FN(oracle_outer_step)(int variant, int bootstrap, int M, int64_t P, int64_t 
             REAL x = load_theta(theta_kind, theta, master, at);
             d[m] = start[at] - x;
         }
-        /* line 8: Delta = (1/M) sum_m Delta_m, summed m = 1..M in order */
-        REAL acc = d[0];
-        for (int m = 1; m < M; ++m) acc = acc + d[m];
+        /* line 8: Delta = (1/M) sum_m Delta_m, summed m = 1..M in order; what is summed is
+           what each worker put on the wire */
+        REAL acc = comm_round(d[0], comm, X, Y, scale[0]);
+        for (int m = 1; m < M; ++m) acc = acc + comm_round(d[m], comm, X, Y, scale[m]);
         REAL D_new = acc / (REAL)M;
 
         if (bootstrap) {
@@ -178,6 +270,21 @@ int FN(oracle_outer_step)(int variant, int bootstrap, int M, int64_t P, int64_t 
     }
     return 0;
 }
+
+/* full-precision communication (the three algorithms as printed) */
+int FN(oracle_outer_step)(int variant, int bootstrap, int M, int64_t P, int64_t stride,
+                          REAL eta, REAL mu, int theta_kind,
+                          void *theta, REAL *master, REAL *start,
+                          REAL *delta_prev_local, REAL *delta_prev_avg, REAL *outer_mom,
+                          int nthreads)
+{
+    return FN(oracle_outer_step_comm)(variant, bootstrap, M, P, stride, eta, mu, theta_kind, theta, master, start,
+                                      delta_prev_local, delta_prev_avg, outer_mom, COMM_F32, 0, 0, NULL, nthreads);
+}
+
+/* exported so that tests can pin the EXMY rounding on its own */
+double FN(oracle_exmy_round)(double y, int X, int Y) { return exmy_round(y, X, Y); }
+double FN(oracle_exmy_max)(int X, int Y) { return exmy_max(X, Y); }
 
 /*
  * The eager outer gradient in the paper's second, equivalent form (Section
