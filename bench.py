@@ -233,7 +233,18 @@ def run_ours(args):
         else:
             grads = inputs.make_grads(M, P, stride, st["gen"], dev, w.grad_kind)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    comm = {"f32": (0, 0, 0), "bf16": (1, 0, 0), "e4m3": (2, 4, 3), "e5m2": (2, 5, 2), "e2m1": (2, 2, 1),
+            "e3m0": (2, 3, 0)}[args.comm]
+    if comm[0]:
+        scratch = torch.zeros(64, dtype=torch.int32, device=dev)
+        state.close()
+        state = binding.State.from_dict(st, H=w.H, outer_lr=w.outer_lr, outer_momentum=w.outer_momentum, beta1=w.beta1,
+                                        beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay, grad_kind=w.grad_kind,
+                                        impl=args.kernel, comm_scratch=scratch)
+    run_outer = (lambda: state.outer_quantized(variant, *comm)) if comm[0] else (lambda: state.outer(variant))
     outer_bpp = outer_bytes_per_param(variant, M, w.theta_kind)
+    if comm[0] == 2:                                    # the max-|Delta_m| pass re-reads theta and start
+        outer_bpp += M * ({0: 4, 1: 2, 2: 4}[w.theta_kind] + 4)
     adam_bpp = adamw_bytes_per_param(M, w.theta_kind, w.grad_kind)
 
     def one_step(timed):
@@ -247,7 +258,7 @@ def run_ours(args):
             for _ in range(w.H):
                 state.inner_adamw(grads, w.inner_lr)
         e1.record()
-        state.outer(variant)
+        run_outer()
         e2.record()
         if not timed:
             return None
@@ -325,7 +336,7 @@ def run_ours(args):
 
     # --- end to end: state in pinned host memory, copies inside the timed region
     e2e = None
-    if args.e2e and not phase:
+    if args.e2e and not phase and not comm[0]:
         keys = ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom")
         need = sum(st[k].numel() * st[k].element_size() for k in keys if st.get(k) is not None)
         try:
@@ -391,7 +402,7 @@ def run_ours(args):
                            "outer_lr": w.outer_lr, "outer_momentum": w.outer_momentum,
                            "l2": "state >> 126 MB L2 and a 256 MB flush write between steps",
                            "sharding": "parameter axis split across ranks, all M replicas of an index on one rank, no collective",
-                           "kernel_impl": ["auto", "direct", "bulk"][args.kernel]},
+                           "kernel_impl": ["auto", "direct", "bulk"][args.kernel], "outer_gradient_wire_format": args.comm},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
                 "replica_params_per_s": value * M, "kernels": kernels or None}
         print(json.dumps(line))
@@ -411,6 +422,8 @@ def main():
     ap.add_argument("--variant", default="eager", choices=["standard", "delayed", "eager"])
     ap.add_argument("--P", type=int, default=0, help="override the workload's parameter count (per GPU)")
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 direct, 2 bulk")
+    ap.add_argument("--comm", default="f32", choices=["f32", "bf16", "e4m3", "e5m2", "e2m1", "e3m0"],
+                    help="wire format of the outer gradients (quantised communication)")
     ap.add_argument("--chunk", type=int, default=64 * 16384, help="elements per chunk of the host-buffer path")
     ap.add_argument("--outer-only", action="store_true", help="phase workloads: time the outer step alone")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false")

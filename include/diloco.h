@@ -65,6 +65,13 @@ enum {
 };
 enum { DILOCO_GRAD_F32 = 0, DILOCO_GRAD_BF16 = 1 };
 
+/* wire format of the outer gradients in diloco_outer_quantized */
+enum {
+  DILOCO_COMM_F32 = 0,  /* full precision: the algorithms as printed */
+  DILOCO_COMM_BF16 = 1, /* bfloat16, round to nearest even, no scaling */
+  DILOCO_COMM_EXMY = 2  /* 1 sign + exp_bits + man_bits float, scaled per replica (see the call) */
+};
+
 /* kernel implementation selector (performance only; results are bit-identical) */
 enum {
   DILOCO_IMPL_AUTO = 0,
@@ -101,6 +108,9 @@ typedef struct {
   float *adam_v;           /* [M, stride] fp32 second moment; NULL if diloco_inner_adamw is not used    */
   uint32_t *device_status; /* 1 word, zero-initialised by the caller; needed only by DILOCO_IMPL_BULK,
                               whose bounded mbarrier waits record a give-up here; else may be NULL      */
+  uint32_t *comm_scratch;  /* [DILOCO_MAX_M] words of scratch, contents irrelevant on entry; needed only by
+                              diloco_outer_quantized with DILOCO_COMM_EXMY (per-replica max |Delta_m|),
+                              else may be NULL                                                            */
 } diloco_buffers_t;
 
 typedef struct diloco_state diloco_state_t; /* opaque, host memory, owned by the library */
@@ -154,6 +164,27 @@ int diloco_outer_delayed(diloco_state_t *state, void *cuda_stream);
  * Errors additionally: BAD_STATE (delta_prev_local or delta_prev_avg missing).
  */
 int diloco_outer_eager(diloco_state_t *state, void *cuda_stream);
+
+/*
+ * Any of the three outer steps with QUANTISED COMMUNICATION of the outer gradients (Section 3,
+ * "Quantized Communication": float32, bfloat16, float8 and float4 "using EXMY").  Only the
+ * operand of the all-reduce is rounded: line 8 becomes Delta = (1/M) sum_m Q_m(Delta_m), while
+ * every local use of Delta_m (line 11's fresh and stale terms, delta_prev_local) keeps fp32.
+ *   DILOCO_COMM_BF16: Q = round to bfloat16 (nearest even).
+ *   DILOCO_COMM_EXMY: Q_m(x) = scale_m * R(x / scale_m), R = nearest number of the float with
+ *     1 sign, exp_bits exponent and man_bits mantissa bits (bias 2^(exp_bits-1) - 1, subnormals,
+ *     every code finite, ties to the even code, saturating), scale_m = max_i |Delta_m[i]| /
+ *     (largest value of the format), or 1 if the replica did not move.  1 <= exp_bits <= 5,
+ *     man_bits >= 0, exp_bits + man_bits <= 7 (E4M3, E5M2: 8 bits; E2M1, E3M0: 4 bits).
+ *     Two kernels: a reduction of max |Delta_m| into comm_scratch (zeroed by the call, so calls
+ *     on one state must not overlap), then the fused step.
+ * variant: 0 standard, 1 delayed, 2 eager; have_prev and the counters advance as in the plain
+ * calls.  DILOCO_COMM_F32 is the plain call.  The paper fixes no bit layout or scaling: the
+ * above is this library's reading.
+ * Errors additionally: INVALID_ARG (format), BAD_STATE (comm_scratch missing for EXMY).
+ */
+int diloco_outer_quantized(diloco_state_t *state, int32_t variant, int32_t comm_format, int32_t exp_bits,
+                           int32_t man_bits, void *cuda_stream);
 
 /*
  * The same three steps restricted to parameter indices [offset, offset + len) of every

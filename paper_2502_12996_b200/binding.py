@@ -18,6 +18,7 @@ THETA_F32, THETA_BF16, THETA_MASTER_BF16 = 0, 1, 2
 GRAD_F32, GRAD_BF16 = 0, 1
 IMPL_AUTO, IMPL_DIRECT, IMPL_BULK = 0, 1, 2
 STANDARD, DELAYED, EAGER = 0, 1, 2
+COMM_F32, COMM_BF16, COMM_EXMY = 0, 1, 2
 MAX_M = 64
 
 
@@ -35,7 +36,7 @@ class Buffers(ctypes.Structure):
     _fields_ = [("theta", ctypes.c_void_p), ("master", ctypes.c_void_p), ("start", ctypes.c_void_p),
                 ("delta_prev_local", ctypes.c_void_p), ("delta_prev_avg", ctypes.c_void_p),
                 ("outer_mom", ctypes.c_void_p), ("adam_m", ctypes.c_void_p), ("adam_v", ctypes.c_void_p),
-                ("device_status", ctypes.c_void_p)]
+                ("device_status", ctypes.c_void_p), ("comm_scratch", ctypes.c_void_p)]
 
 
 class DilocoError(RuntimeError):
@@ -56,6 +57,7 @@ SYMBOLS = {
     "diloco_outer_standard": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_outer_delayed": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_outer_eager": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_outer_quantized": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
     "diloco_outer_fragment": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
     "diloco_outer_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Buffers), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int64]),
     "diloco_state_get_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)]),
@@ -115,22 +117,23 @@ def _stream_ptr(stream) -> Optional[int]:
 
 
 def make_buffers(theta=None, master=None, start=None, delta_prev_local=None, delta_prev_avg=None, outer_mom=None,
-                 adam_m=None, adam_v=None, device_status=None) -> Buffers:
+                 adam_m=None, adam_v=None, device_status=None, comm_scratch=None) -> Buffers:
     return Buffers(_ptr(theta), _ptr(master), _ptr(start), _ptr(delta_prev_local), _ptr(delta_prev_avg),
-                   _ptr(outer_mom), _ptr(adam_m), _ptr(adam_v), _ptr(device_status))
+                   _ptr(outer_mom), _ptr(adam_m), _ptr(adam_v), _ptr(device_status), _ptr(comm_scratch))
 
 
 class State:
     """Owns a diloco_state_t handle and keeps the borrowed tensors alive."""
 
     def __init__(self, *, M, P, stride, theta, start, outer_mom, master=None, delta_prev_local=None,
-                 delta_prev_avg=None, adam_m=None, adam_v=None, device_status=None, H=0, outer_lr=0.7,
+                 delta_prev_avg=None, adam_m=None, adam_v=None, device_status=None, comm_scratch=None, H=0,
+                 outer_lr=0.7,
                  outer_momentum=0.9, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1, theta_kind=THETA_F32,
                  grad_kind=GRAD_F32, have_prev=1, impl=IMPL_AUTO):
         self._handle = ctypes.c_void_p()
         self.tensors = dict(theta=theta, master=master, start=start, delta_prev_local=delta_prev_local,
                             delta_prev_avg=delta_prev_avg, outer_mom=outer_mom, adam_m=adam_m, adam_v=adam_v,
-                            device_status=device_status)
+                            device_status=device_status, comm_scratch=comm_scratch)
         self.config = Config(M, H, P, stride, outer_lr, outer_momentum, beta1, beta2, eps, weight_decay,
                              theta_kind, grad_kind, int(have_prev), impl)
         self.buffers = make_buffers(**self.tensors)
@@ -171,6 +174,10 @@ class State:
 
     def outer(self, variant: int, stream=None) -> None:
         (self.outer_standard, self.outer_delayed, self.outer_eager)[variant](stream)
+
+    def outer_quantized(self, variant, comm_format, exp_bits=0, man_bits=0, stream=None) -> None:
+        _check(load_library().diloco_outer_quantized(self._handle, variant, comm_format, exp_bits, man_bits,
+                                                     _stream_ptr(stream)), "diloco_outer_quantized")
 
     def outer_fragment(self, variant, bootstrap, offset, length, stream=None) -> None:
         _check(load_library().diloco_outer_fragment(self._handle, variant, int(bool(bootstrap)), offset, length,

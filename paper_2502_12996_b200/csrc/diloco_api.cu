@@ -70,10 +70,11 @@ int validate_buffers(const diloco_config_t *c, const diloco_buffers_t *b) {
   for (const void *p : all)
     if (p && !aligned16(p)) return DILOCO_ERR_MISALIGNED;
   if (b->device_status && (reinterpret_cast<uintptr_t>(b->device_status) & 3u)) return DILOCO_ERR_MISALIGNED;
+  if (b->comm_scratch && (reinterpret_cast<uintptr_t>(b->comm_scratch) & 3u)) return DILOCO_ERR_MISALIGNED;
   return DILOCO_OK;
 }
 
-template <int M, int G, int VAR, int TK, bool BOOT, int V, int NT, int MINB>
+template <int M, int G, int VAR, int TK, bool BOOT, int V, int NT, int MINB, bool Q>
 int launch_outer_t(const OuterArgs &a, cudaStream_t s) {
   constexpr int CW = 32 / G;
   const long long nvec = a.P / V;
@@ -81,19 +82,19 @@ int launch_outer_t(const OuterArgs &a, cudaStream_t s) {
   long long blocks = (warps * 32 + NT - 1) / NT;
   if (blocks < 1) blocks = 1; // the last block also handles the P % V tail
   if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
-  outer_step_kernel<M, G, VAR, TK, BOOT, V, NT, MINB><<<(unsigned)blocks, NT, 0, s>>>(a);
+  outer_step_kernel<M, G, VAR, TK, BOOT, V, NT, MINB, Q><<<(unsigned)blocks, NT, 0, s>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1);
   return DILOCO_OK;
 }
 
-template <int M, int G, int V, int NT, int MINB>
+template <bool Q, int M, int G, int V, int NT, int MINB>
 int launch_outer_m(int var, int tk, bool boot, const OuterArgs &a, cudaStream_t s) {
 #define DILOCO_CASE(VAR_, TK_)                                                                           \
   if (var == VAR_ && tk == TK_) {                                                                        \
-    if (VAR_ != VAR_STANDARD && boot) return launch_outer_t<M, G, VAR_, TK_, true, V, NT, MINB>(a, s);   \
-    return launch_outer_t<M, G, VAR_, TK_, false, V, NT, MINB>(a, s);                                    \
+    if (VAR_ != VAR_STANDARD && boot) return launch_outer_t<M, G, VAR_, TK_, true, V, NT, MINB, Q>(a, s); \
+    return launch_outer_t<M, G, VAR_, TK_, false, V, NT, MINB, Q>(a, s);                                  \
   }
   DILOCO_CASE(VAR_STANDARD, TK_F32)
   DILOCO_CASE(VAR_STANDARD, TK_BF16)
@@ -112,19 +113,20 @@ int launch_outer_m(int var, int tk, bool boot, const OuterArgs &a, cudaStream_t 
 // chosen by measurement on B200 under two rules: no register spills, and every warp-level
 // access covers at least 128 contiguous bytes of a row (64-byte runs halved the bandwidth).
 // M <= 3: one thread per column.  M = 4, 8, 16: the replica axis is split over G lanes.
+template <bool Q>
 int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterArgs &a, cudaStream_t s) {
   const int tk = st->cfg.theta_kind;
   switch (st->cfg.M) {
-    case 1: return launch_outer_m<1, 1, 4, 128, 8>(var, tk, boot, a, s);
-    case 2: return launch_outer_m<2, 1, 4, 128, 6>(var, tk, boot, a, s);
-    case 3: return launch_outer_m<3, 1, 4, 128, 4>(var, tk, boot, a, s);
-    case 4: return launch_outer_m<4, 2, 4, 128, 8>(var, tk, boot, a, s);
+    case 1: return launch_outer_m<Q, 1, 1, 4, 128, 8>(var, tk, boot, a, s);
+    case 2: return launch_outer_m<Q, 2, 1, 4, 128, 6>(var, tk, boot, a, s);
+    case 3: return launch_outer_m<Q, 3, 1, 4, 128, 4>(var, tk, boot, a, s);
+    case 4: return launch_outer_m<Q, 4, 2, 4, 128, 8>(var, tk, boot, a, s);
     case 8:
       // fp32 rows: 16 lanes x 8 B = 128 B per row; bf16 rows need the wider vector for that
-      if (tk == TK_F32) return launch_outer_m<8, 2, 2, 256, 3>(var, tk, boot, a, s);
-      return launch_outer_m<8, 2, 4, 128, 4>(var, tk, boot, a, s);
-    case 16: return launch_outer_m<16, 4, 4, 128, 4>(var, tk, boot, a, s);
-    default: return launch_outer_m<0, 1, 4, 128, 4>(var, tk, boot, a, s);
+      if (tk == TK_F32) return launch_outer_m<Q, 8, 2, 2, 256, 3>(var, tk, boot, a, s);
+      return launch_outer_m<Q, 8, 2, 4, 128, 4>(var, tk, boot, a, s);
+    case 16: return launch_outer_m<Q, 16, 4, 4, 128, 4>(var, tk, boot, a, s);
+    default: return launch_outer_m<Q, 0, 1, 4, 128, 4>(var, tk, boot, a, s);
   }
 }
 
@@ -151,7 +153,52 @@ OuterArgs outer_args(const diloco_state *st, int64_t offset, int64_t len) {
   a.mu = st->cfg.outer_momentum;
   a.fM = (float)st->cfg.M;
   a.M = st->cfg.M;
+  a.amax = nullptr;
+  a.fmt_max = 0.f;
+  a.comm = COMM_F32;
+  a.man_bits = a.emin = a.bias = 0;
   return a;
+}
+
+template <int TK>
+int launch_amax_t(const diloco_state *st, const OuterArgs &a, unsigned *amax, cudaStream_t s) {
+  constexpr int NT = 256, U = 4;
+  const long long nvec = a.P / 4;
+  long long blocks = (nvec + (long long)NT * U - 1) / ((long long)NT * U);
+  const long long cap = (long long)st->sm_count * 8; // grid-stride: few atomics, every SM busy
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  dim3 grid((unsigned)blocks, (unsigned)st->cfg.M);
+  delta_amax_kernel<TK, NT, U><<<grid, NT, 0, s>>>(a, amax);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1);
+  return DILOCO_OK;
+}
+
+// One quantised outer step on indices [0, P): (EXMY only) zero the per-replica maxima and
+// reduce max |Delta_m| into `scratch`, then the fused step with the wire rounding in line 8.
+int launch_outer_quantized(diloco_state *st, int var, bool boot, int comm, int X, int Y, unsigned *scratch,
+                           cudaStream_t s) {
+  OuterArgs a = outer_args(st, 0, st->cfg.P);
+  a.comm = comm;
+  if (comm == COMM_EXMY) {
+    a.bias = (1 << (X - 1)) - 1;
+    a.emin = 1 - a.bias;
+    a.man_bits = Y;
+    a.fmt_max = std::ldexp(2.0f - std::ldexp(1.0f, -Y), (1 << X) - 1 - a.bias);
+    a.amax = scratch;
+    cudaError_t e = cudaMemsetAsync(scratch, 0, sizeof(unsigned) * (size_t)st->cfg.M, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int rc;
+    switch (st->cfg.theta_kind) {
+      case TK_F32: rc = launch_amax_t<TK_F32>(st, a, scratch, s); break;
+      case TK_BF16: rc = launch_amax_t<TK_BF16>(st, a, scratch, s); break;
+      default: rc = launch_amax_t<TK_MASTER_BF16>(st, a, scratch, s); break;
+    }
+    if (rc != DILOCO_OK) return rc;
+  }
+  return launch_outer_direct<true>(st, var, boot, a, s);
 }
 
 // Bulk (TMA-staged) form: one CTA ring per SM slot, grid capped by the tile count.
@@ -202,7 +249,7 @@ int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t l
     if (st->cfg.M == 2 && len >= 1024) return launch_bulk_m<2, 1024, 3, 256>(st, var, st->cfg.theta_kind, a, s);
     if (st->cfg.M == 4 && len >= 512) return launch_bulk_m<4, 512, 3, 128>(st, var, st->cfg.theta_kind, a, s);
   }
-  return launch_outer_direct(st, var, boot, a, s);
+  return launch_outer_direct<false>(st, var, boot, a, s);
 }
 
 int outer_whole(diloco_state *st, int var, void *stream) {
@@ -315,6 +362,26 @@ int diloco_inner_adamw(diloco_state_t *st, const void *grads, int64_t grad_strid
 int diloco_outer_standard(diloco_state_t *st, void *stream) { return outer_whole(st, VAR_STANDARD, stream); }
 int diloco_outer_delayed(diloco_state_t *st, void *stream) { return outer_whole(st, VAR_DELAYED, stream); }
 int diloco_outer_eager(diloco_state_t *st, void *stream) { return outer_whole(st, VAR_EAGER, stream); }
+
+int diloco_outer_quantized(diloco_state_t *st, int32_t variant, int32_t comm_format, int32_t exp_bits, int32_t man_bits,
+                           void *stream) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  int rc = check_variant(st, variant);
+  if (rc != DILOCO_OK) return rc;
+  if (comm_format == DILOCO_COMM_F32) return outer_whole(st, variant, stream);
+  if (comm_format != DILOCO_COMM_BF16 && comm_format != DILOCO_COMM_EXMY) return DILOCO_ERR_INVALID_ARG;
+  if (comm_format == DILOCO_COMM_EXMY) {
+    if (exp_bits < 1 || exp_bits > 5 || man_bits < 0 || exp_bits + man_bits > 7) return DILOCO_ERR_INVALID_ARG;
+    if (!st->buf.comm_scratch) return DILOCO_ERR_BAD_STATE;
+  }
+  const bool boot = (variant != VAR_STANDARD) && st->have_prev == 0;
+  rc = launch_outer_quantized(st, variant, boot, comm_format, exp_bits, man_bits, st->buf.comm_scratch,
+                              static_cast<cudaStream_t>(stream));
+  if (rc != DILOCO_OK) return rc;
+  if (variant != VAR_STANDARD) st->have_prev = 1;
+  st->outer_step += 1;
+  return DILOCO_OK;
+}
 
 int diloco_outer_fragment(diloco_state_t *st, int32_t variant, int32_t bootstrap, int64_t offset, int64_t len,
                           void *stream) {

@@ -31,7 +31,16 @@ struct OuterArgs {
   long long stride; // elements between replicas
   float eta, mu, fM;
   int M;            // used by the runtime-M kernel only
+  // quantised communication of the outer gradients (Q kernels only)
+  const unsigned *amax; // [M] bit patterns of max_i |Delta_m[i]|, written by delta_amax_kernel
+  float fmt_max;        // largest EXMY value
+  int comm;             // COMM_BF16 or COMM_EXMY
+  int man_bits;         // Y
+  int emin;             // 1 - bias: exponent of the smallest normal
+  int bias;             // 2^(X-1) - 1
 };
+
+enum { COMM_F32 = 0, COMM_BF16 = 1, COMM_EXMY = 2 };
 
 struct AdamArgs {
   void *theta;
@@ -156,6 +165,85 @@ __device__ __forceinline__ void nesterov(float g, float eta, float mu, float &b,
   b = nb;
 }
 
+// ---------------------------------------------------------------- wire formats of Delta_m
+// Section 3, "Quantized Communication": the all-reduce operand is rounded to bfloat16 or to
+// an EXMY float (1 sign, X exponent, Y mantissa bits, bias 2^(X-1)-1, subnormals, every code
+// finite, round to nearest with ties to the even code, saturating) after scaling each
+// replica's vector so that its largest magnitude lands on the format's largest value.
+// All scalings below are by powers of two and therefore exact in fp32.
+__device__ __forceinline__ float exmy_round(float y, const OuterArgs &a) {
+  const float ay = fabsf(y);
+  if (ay == 0.f) return y;
+  int E = (int)((__float_as_uint(ay) >> 23) & 0xffu) - 127; // binade of |y| (fp32 subnormals: clamped next)
+  E = max(E, a.emin);                                       // below the smallest normal the spacing is fixed
+  const int qe = E - a.man_bits;                            // spacing = 2^qe
+  const float n = ay * __uint_as_float((unsigned)(127 - qe) << 23); // |y| / spacing, exact
+  float r = rintf(n);                                       // halves go to the even integer = even code ...
+  if (a.man_bits == 0 && n == 1.5f) r = ((E + a.bias) & 1) ? 2.f : 1.f; // ... except with no mantissa bits,
+                                                            // where the code's parity is the exponent field's
+  float q = r * __uint_as_float((unsigned)(127 + qe) << 23);
+  q = fminf(q, a.fmt_max);
+  return copysignf(q, y);
+}
+
+// the per-replica scale: max |Delta_m| maps to the format's largest value (1 if the replica did not move)
+__device__ __forceinline__ float comm_scale(const OuterArgs &a, int m) {
+  if (a.comm != COMM_EXMY) return 1.f;
+  const float amax = __uint_as_float(a.amax[m]);
+  return amax > 0.f ? amax / a.fmt_max : 1.f;
+}
+
+// what replica m puts on the wire for one element of its outer gradient
+__device__ __forceinline__ float comm_round(float d, float scale, const OuterArgs &a) {
+  if (a.comm == COMM_BF16) return bf16_bits_to_f32(f32_to_bf16_bits(d));
+  const float y = d / scale;
+  return exmy_round(y, a) * scale;
+}
+
+// Pass 1 of a quantised step: amax[m] = max_i |s_m[i] - theta_m[i]| (fp32, exact: max is
+// order-free).  grid = (blocks, M); non-negative floats order like their bit patterns.
+template <int TK, int NT, int U>
+__global__ void __launch_bounds__(NT) delta_amax_kernel(const OuterArgs a, unsigned *amax) {
+  const int m = blockIdx.y;
+  const long long nvec = a.P / 4;
+  float best = 0.f;
+  for (long long j0 = (long long)blockIdx.x * (NT * U) + threadIdx.x; j0 < nvec; j0 += (long long)gridDim.x * (NT * U)) {
+    float s[U][4], x[U][4];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const long long j = j0 + (long long)u * NT;
+      if (j < nvec) {
+        F32Vec<4>::load(a.start + m * a.stride + j * 4, s[u]);
+        load_theta<TK, 4>(a, m * a.stride + j * 4, x[u]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[u][e] = x[u][e] = 0.f;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) best = fmaxf(best, fabsf(s[u][e] - x[u][e]));
+  }
+  if (blockIdx.x == 0) {
+    for (long long i = nvec * 4 + threadIdx.x; i < a.P; i += NT) {
+      float s[1], x[1];
+      F32Vec<1>::load(a.start + m * a.stride + i, s);
+      load_theta<TK, 1>(a, m * a.stride + i, x);
+      best = fmaxf(best, fabsf(s[0] - x[0]));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
+  __shared__ float warp_best[NT / 32];
+  if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < NT / 32; ++w) best = fmaxf(best, warp_best[w]);
+    atomicMax(amax + m, __float_as_uint(best));
+  }
+}
+
 // ---------------------------------------------------------------- outer step, compile-time M
 // One column = V consecutive parameter indices.  A thread owns R = M / G replicas
 // (m0 .. m0+R-1) of its column; with G > 1 the G lanes that share a column sit CW = 32 / G
@@ -163,10 +251,11 @@ __device__ __forceinline__ void nesterov(float g, float eta, float mu, float &b,
 // to group with shuffles, so the mean is still the left-to-right sum m = 0 .. M-1 and every
 // lane divides the same total (identical bits in all G lanes).  Splitting the replica axis
 // keeps the per-thread register count of M = 8 .. 64 at that of M = 4.
-template <int R, int G, int VAR, int TK, bool BOOT, int V>
+template <int R, int G, int VAR, int TK, bool BOOT, int V, bool Q = false>
 __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, int m0, bool active) {
   constexpr int CW = 32 / G;
   float s[R][V], d[R][V], b[R][V], pl[R][V], pa[V], mean[V];
+  float w[R][V]; // what replica m0+r sends into the all-reduce: Delta_m, or its wire-format rounding
   if (active) {
     // Alg. 1-3 line 7 operands: theta_m^(t-H) and theta_m^(t)
 #pragma unroll
@@ -194,13 +283,19 @@ __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, in
       x[r][e] = d[r][e];
       d[r][e] = s[r][e] - d[r][e]; // line 7: Delta_m
     }
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const float scale = Q ? comm_scale(a, m0 + r) : 1.f;
+#pragma unroll
+    for (int e = 0; e < V; ++e) w[r][e] = Q ? comm_round(d[r][e], scale, a) : d[r][e];
+  }
   // line 8: Delta = (1/M) sum_m Delta_m, m in order (stands in for the all-reduce)
   if (G == 1) {
 #pragma unroll
     for (int e = 0; e < V; ++e) {
-      mean[e] = d[0][e];
+      mean[e] = w[0][e];
 #pragma unroll
-      for (int r = 1; r < R; ++r) mean[e] = mean[e] + d[r][e];
+      for (int r = 1; r < R; ++r) mean[e] = mean[e] + w[r][e];
     }
   } else {
     const int g = (threadIdx.x & 31) / CW;
@@ -212,9 +307,9 @@ __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, in
       for (int e = 0; e < V; ++e) {
         const float prev = __shfl_up_sync(0xffffffffu, mean[e], CW); // running sum of groups < gg
         if (g == gg) {
-          float acc = (gg == 0) ? d[0][e] : prev + d[0][e];
+          float acc = (gg == 0) ? w[0][e] : prev + w[0][e];
 #pragma unroll
-          for (int r = 1; r < R; ++r) acc = acc + d[r][e];
+          for (int r = 1; r < R; ++r) acc = acc + w[r][e];
           mean[e] = acc;
         }
       }
@@ -265,16 +360,18 @@ __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, in
 // ---------------------------------------------------------------- outer step, runtime M
 // Two sweeps over the replicas: the first forms the mean, the second re-reads s_m and
 // theta_m (L1/L2 hits: the same thread read them a few hundred cycles earlier) and updates.
-template <int VAR, int TK, bool BOOT, int V>
+template <int VAR, int TK, bool BOOT, int V, bool Q = false>
 __device__ __forceinline__ void outer_column_rt(const OuterArgs &a, long long i) {
   float mean[V];
   for (int m = 0; m < a.M; ++m) {
     float s[V], x[V];
     F32Vec<V>::load_cached(a.start + m * a.stride + i, s);
     load_theta<TK, V>(a, m * a.stride + i, x, true);
+    const float scale = Q ? comm_scale(a, m) : 1.f;
 #pragma unroll
     for (int e = 0; e < V; ++e) {
       float dm = s[e] - x[e];
+      if (Q) dm = comm_round(dm, scale, a);
       mean[e] = (m == 0) ? dm : mean[e] + dm;
     }
   }
@@ -323,7 +420,7 @@ __device__ __forceinline__ void outer_column_rt(const OuterArgs &a, long long i)
 // persistent grid-stride loop.  M = 0 selects the runtime-M form (G = 1).
 // Grid: ceil(ceil(nvec / CW) * 32 / NT) blocks, nvec = P / V, CW = 32 / G.  The ragged tail
 // (P % V indices) is done one index per thread by the last block with the runtime-M code.
-template <int M, int G, int VAR, int TK, bool BOOT, int V, int NT, int MINB>
+template <int M, int G, int VAR, int TK, bool BOOT, int V, int NT, int MINB, bool Q = false>
 __global__ void __launch_bounds__(NT, MINB) outer_step_kernel(const OuterArgs a) {
   constexpr int CW = 32 / G;
   const long long nvec = a.P / V;
@@ -333,13 +430,13 @@ __global__ void __launch_bounds__(NT, MINB) outer_step_kernel(const OuterArgs a)
   if (M > 0) {
     constexpr int R = (M > 0 ? M : 1) / G;
     const bool active = j < nvec;
-    if (G > 1 || active) outer_column<R, G, VAR, TK, BOOT, V>(a, j * V, (lane / CW) * R, active);
+    if (G > 1 || active) outer_column<R, G, VAR, TK, BOOT, V, Q>(a, j * V, (lane / CW) * R, active);
   } else {
-    if (j < nvec) outer_column_rt<VAR, TK, BOOT, V>(a, j * V);
+    if (j < nvec) outer_column_rt<VAR, TK, BOOT, V, Q>(a, j * V);
   }
   if (blockIdx.x == gridDim.x - 1) {
     const long long i = nvec * V + threadIdx.x;
-    if (i < a.P) outer_column_rt<VAR, TK, BOOT, 1>(a, i);
+    if (i < a.P) outer_column_rt<VAR, TK, BOOT, 1, Q>(a, i);
   }
 }
 

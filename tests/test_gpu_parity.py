@@ -131,6 +131,57 @@ def test_worked_example_on_gpu():
         state.close()
 
 
+# ---------------------------------------------------------------- quantised communication
+FORMATS = {"bf16": (binding.COMM_BF16, 0, 0), "e4m3": (binding.COMM_EXMY, 4, 3), "e5m2": (binding.COMM_EXMY, 5, 2),
+           "e2m1": (binding.COMM_EXMY, 2, 1), "e3m0": (binding.COMM_EXMY, 3, 0)}
+
+
+@pytest.mark.parametrize("fmt", list(FORMATS))
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("M,P,theta_kind", [(2, 100_003, 0), (4, 300_001, 0), (4, 70_001, 1), (8, 50_002, 2),
+                                            (16, 40_001, 0), (5, 20_003, 0), (1, 9_999, 0)])
+def test_quantized_communication(oracle, fmt, variant, M, P, theta_kind):
+    """The all-reduce operand rounded to bf16 / scaled EXMY: per-replica maxima reduced on the
+    device, same scale, same rounding (ties included), same bits as the oracle; first call is
+    the t = H bootstrap, then two regular steps."""
+    comm, X, Y = FORMATS[fmt]
+    st, checks = make(M, P, 1700 + M, theta_kind)
+    h = host_copy(st)
+    scratch = torch.full((64,), 0x7fffffff, dtype=torch.int32, device=DEV)     # stale contents must not matter
+    state = binding.State.from_dict(st, have_prev=0, comm_scratch=scratch)
+    for k in range(3):
+        if k:
+            inputs.inner_phase_standin(st)
+            h["theta"] = to_numpy(st["theta"])
+            h["master"] = to_numpy(st["master"])
+        state.outer_quantized(variant, comm, X, Y)
+        oracle.outer_step(variant, M=M, P=P, stride=st["stride"], eta=0.7, mu=0.9, theta=h["theta"], start=h["start"],
+                          outer_mom=h["outer_mom"], delta_prev_local=h["delta_prev_local"],
+                          delta_prev_avg=h["delta_prev_avg"], master=h["master"], theta_kind=theta_kind,
+                          bootstrap=(variant != 0 and k == 0), comm=comm, exp_bits=X, man_bits=Y, nthreads=8)
+        torch.cuda.synchronize()
+        assert_state_equal(st, h, what=f"quantised {fmt} {NAMES[variant]} M={M} step {k + 1}")
+    for c in checks:
+        c()
+    assert state.get_counters()[1] == 3
+
+
+def test_quantized_argument_checks():
+    st, _ = make(2, 1000, 1800, 0, guards=False)
+    state = binding.State.from_dict(st)                        # no comm_scratch
+    with pytest.raises(binding.DilocoError) as e:
+        state.outer_quantized(2, binding.COMM_EXMY, 4, 3)
+    assert e.value.status == binding.ERR_BAD_STATE
+    state.outer_quantized(2, binding.COMM_BF16)                 # bf16 needs no scratch
+    for X, Y in ((0, 3), (6, 1), (4, 4), (3, -1)):
+        with pytest.raises(binding.DilocoError) as e:
+            state.outer_quantized(2, binding.COMM_EXMY, X, Y)
+        assert e.value.status == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.DilocoError):
+        state.outer_quantized(2, 7)
+    torch.cuda.synchronize()
+
+
 # ---------------------------------------------------------------- inner AdamW
 def run_adamw(oracle, M, P, theta_kind, grad_kind, steps, seed, segments=0):
     st, checks = make(M, P, seed, theta_kind, with_adam=True)
