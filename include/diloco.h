@@ -187,6 +187,34 @@ int diloco_outer_quantized(diloco_state_t *state, int32_t variant, int32_t comm_
                            int32_t man_bits, void *cuda_stream);
 
 /*
+ * diloco_outer_quantized for callers that cannot provide comm_scratch.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, same arithmetic, same results.)
+ *
+ * Who needs it: code that gets handed the state tensors and nothing else and has no way to
+ * obtain one more device buffer - for instance an extension running inside a trainer whose
+ * memory pool already owns all of the GPU's memory, so that a raw cudaMalloc fails, or a
+ * callback that must not allocate because allocation may synchronise the device.  For them
+ * the per-replica maxima are reduced into an array that is part of the library image
+ * instead: DILOCO_MAX_M (64) words = 256 bytes of device memory, present on every GPU that
+ * loads the library for as long as the process lives.  The state's comm_scratch is ignored
+ * and may be NULL.  The call allocates and frees nothing, on the host side of CUDA or on the
+ * device.
+ *
+ * Limits and rules:
+ *   - M <= DILOCO_MAX_M, else DILOCO_ERR_UNSUPPORTED (one word of scratch per replica).
+ *   - the state's device must be the current device, else DILOCO_ERR_BAD_STATE.
+ *   - the first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress) and keeps it; make that first call outside any stream capture.
+ *   - all states and all calls on a device share the one array.  The call clears the words
+ *     it uses before reducing into them, so stale contents never matter, but two calls whose
+ *     kernels can overlap on the GPU (different streams, no ordering between them) race on
+ *     it: order such calls yourself.
+ * Otherwise identical to diloco_outer_quantized, including errors, have_prev and counters.
+ */
+int diloco_outer_quantized_static(diloco_state_t *state, int32_t variant, int32_t comm_format, int32_t exp_bits,
+                                  int32_t man_bits, void *cuda_stream);
+
+/*
  * The same three steps restricted to parameter indices [offset, offset + len) of every
  * replica (a fragment, as Streaming DiLoCo applies the outer step to parts of the model
  * on different schedules, Section 3).  variant: 0 standard, 1 delayed, 2 eager.  bootstrap

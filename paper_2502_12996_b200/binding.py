@@ -58,6 +58,7 @@ SYMBOLS = {
     "diloco_outer_delayed": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_outer_eager": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_outer_quantized": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
+    "diloco_outer_quantized_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
     "diloco_outer_fragment": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
     "diloco_outer_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Buffers), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int64]),
     "diloco_state_get_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)]),
@@ -178,6 +179,11 @@ class State:
     def outer_quantized(self, variant, comm_format, exp_bits=0, man_bits=0, stream=None) -> None:
         _check(load_library().diloco_outer_quantized(self._handle, variant, comm_format, exp_bits, man_bits,
                                                      _stream_ptr(stream)), "diloco_outer_quantized")
+
+    def outer_quantized_static(self, variant, comm_format, exp_bits=0, man_bits=0, stream=None) -> None:
+        """diloco_outer_quantized with the scratch inside the library (no comm_scratch needed)."""
+        _check(load_library().diloco_outer_quantized_static(self._handle, variant, comm_format, exp_bits, man_bits,
+                                                            _stream_ptr(stream)), "diloco_outer_quantized_static")
 
     def outer_fragment(self, variant, bootstrap, offset, length, stream=None) -> None:
         _check(load_library().diloco_outer_fragment(self._handle, variant, int(bool(bootstrap)), offset, length,

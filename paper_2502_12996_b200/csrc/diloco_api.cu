@@ -8,6 +8,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -27,6 +28,11 @@ struct diloco_state {
   std::vector<cudaEvent_t> events; // host-path chunk events, created on first use
   cudaEvent_t last_d2h;
 };
+
+// Scratch of diloco_outer_quantized_static: part of the library image, so every GPU that loads
+// the library holds these 64 words (256 bytes) until the process exits.
+constexpr int kStaticScratchWords = DILOCO_MAX_M;
+static __device__ __align__(256) unsigned g_static_scratch[kStaticScratchWords];
 
 namespace {
 
@@ -279,6 +285,26 @@ int launch_adamw_t(const diloco_state *st, const AdamArgs &a, cudaStream_t s) {
   return DILOCO_OK;
 }
 
+// ---- per-device address of the scratch inside the library image ----------------------------
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned *g_static_ptr[kMaxDevices] = {}; // device address of g_static_scratch, per device ordinal
+
+// `g_static_scratch` in host code is only a handle for the runtime, not a device address:
+// ask the runtime for the address on the device that is current, once per device.
+int static_scratch_for_current_device(int device, unsigned **out) {
+  if (device < 0 || device >= kMaxDevices) return DILOCO_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[device]) {
+    void *p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_static_ptr[device] = static_cast<unsigned *>(p);
+  }
+  *out = g_static_ptr[device];
+  return DILOCO_OK;
+}
+
 } // namespace
 
 extern "C" {
@@ -376,6 +402,34 @@ int diloco_outer_quantized(diloco_state_t *st, int32_t variant, int32_t comm_for
   }
   const bool boot = (variant != VAR_STANDARD) && st->have_prev == 0;
   rc = launch_outer_quantized(st, variant, boot, comm_format, exp_bits, man_bits, st->buf.comm_scratch,
+                              static_cast<cudaStream_t>(stream));
+  if (rc != DILOCO_OK) return rc;
+  if (variant != VAR_STANDARD) st->have_prev = 1;
+  st->outer_step += 1;
+  return DILOCO_OK;
+}
+
+int diloco_outer_quantized_static(diloco_state_t *st, int32_t variant, int32_t comm_format, int32_t exp_bits,
+                                  int32_t man_bits, void *stream) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  int rc = check_variant(st, variant);
+  if (rc != DILOCO_OK) return rc;
+  if (comm_format < DILOCO_COMM_F32 || comm_format > DILOCO_COMM_EXMY) return DILOCO_ERR_INVALID_ARG;
+  if (comm_format == DILOCO_COMM_EXMY &&
+      (exp_bits < 1 || exp_bits > 5 || man_bits < 0 || exp_bits + man_bits > 7))
+    return DILOCO_ERR_INVALID_ARG;
+  if (st->cfg.M > kStaticScratchWords) return DILOCO_ERR_UNSUPPORTED; // one word of scratch per replica
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev != st->device) return DILOCO_ERR_BAD_STATE; // the state's GPU must be the current one
+  unsigned *scratch = nullptr;
+  rc = static_scratch_for_current_device(dev, &scratch);
+  if (rc != DILOCO_OK) return rc;
+  if (comm_format == DILOCO_COMM_F32) return outer_whole(st, variant, stream);
+  const bool boot = (variant != VAR_STANDARD) && st->have_prev == 0;
+  // launch_outer_quantized zeroes the M words it reduces into before every use
+  rc = launch_outer_quantized(st, variant, boot, comm_format, exp_bits, man_bits, scratch,
                               static_cast<cudaStream_t>(stream));
   if (rc != DILOCO_OK) return rc;
   if (variant != VAR_STANDARD) st->have_prev = 1;
