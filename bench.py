@@ -216,6 +216,9 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     w = inputs.WORKLOADS[args.workload]
     P = args.P or w.P                                       # per GPU: weak scaling, every rank the full shape
+    if args.strong:                                         # total work fixed: this rank's 64-aligned range
+        lo, hi = shard_bounds(P, world, rank)
+        P = hi - lo
     variant = {"standard": 0, "delayed": 1, "eager": 2}[args.variant]
     M = w.M
     phase = w.H > 0 and not args.outer_only
@@ -290,7 +293,13 @@ def run_ours(args):
         l = torch.tensor([launches], device=dev)
         dist.all_reduce(l)
         launches = int(l[0])
-    value = world * P / (step_ms * 1e-3)
+    P_job = P * world
+    if args.strong:
+        t = torch.tensor([P], device=dev, dtype=torch.int64)
+        if world > 1:
+            dist.all_reduce(t)
+        P_job = int(t[0])
+    value = P_job / (step_ms * 1e-3)
 
     # --- roofline of the dominant kernel
     peak, peak_kind = load_peak()
@@ -368,7 +377,7 @@ def run_ours(args):
                     and not (k == "delta_prev_avg" and variant == 0)]
             h2d = sum(leg_bytes(k) for k in used if not (k == "theta" and w.theta_kind == 2))
             d2h = sum(leg_bytes(k) for k in used)
-            e2e = {"value": world * P / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            e2e = {"value": P_job / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                    "ms_per_step": e_ms, "chunk": args.chunk, "timing": "host clock around the call + stream sync",
                    "pcie_GBps_each_way": h2d / e_ms / 1e6}
             del pinned
@@ -394,7 +403,7 @@ def run_ours(args):
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-                "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "ms_per_step": step_ms, "higher_is_better": True, "scaling": "strong" if args.strong else "weak", "vs_baseline": None,
                 "dtype": "f32", "data": "synthetic",
                 "config": {"workload": args.workload, "variant": args.variant, "M": M, "P_per_gpu": P,
                            "theta": ["f32", "bf16", "f32 master + bf16 copy"][w.theta_kind],
@@ -425,6 +434,7 @@ def main():
     ap.add_argument("--comm", default="f32", choices=["f32", "bf16", "e4m3", "e5m2", "e2m1", "e3m0"],
                     help="wire format of the outer gradients (quantised communication)")
     ap.add_argument("--chunk", type=int, default=64 * 16384, help="elements per chunk of the host-buffer path")
+    ap.add_argument("--strong", action="store_true", help="split the workload's P across ranks instead of one full shape per rank")
     ap.add_argument("--outer-only", action="store_true", help="phase workloads: time the outer step alone")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")

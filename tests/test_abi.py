@@ -122,3 +122,12 @@ def test_product_does_not_import_the_oracle():
     pat = re.compile(r"^\s*(import\s+oracle|from\s+oracle|from\s+\.+\s*oracle)|libdiloco_oracle|oracle/|#include.*oracle", re.M)
     for f in list(pkg.rglob("*.py")) + list(pkg.rglob("*.cu")) + list(pkg.rglob("*.cuh")):
         assert not pat.search(f.read_text()), f
+
+
+def test_no_kernel_spills_registers(lib):
+    """Design rule found by measurement: a kernel that spills even a few bytes loses a third of
+    its bandwidth, so every launch shape is chosen to compile without spills or stack frames."""
+    res = build.kernel_resources()
+    assert len(res) > 100
+    bad = [(n, r, s, st) for n, r, s, st in res if s > 0 or st > 0]
+    assert not bad, bad
