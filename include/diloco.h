@@ -46,6 +46,7 @@ extern "C" {
 #endif
 
 #define DILOCO_MAX_M 64
+#define DILOCO_MAX_OVERLAP 4
 
 enum {
   DILOCO_OK = 0,
@@ -91,18 +92,28 @@ typedef struct {
   float weight_decay;   /* AdamW, decoupled, >= 0 */
   int32_t theta_kind;   /* DILOCO_THETA_* */
   int32_t grad_kind;    /* DILOCO_GRAD_* : dtype of the grads argument of diloco_inner_adamw */
-  int32_t have_prev;    /* 1: delta_prev_local / delta_prev_avg already hold the previous phase's
-                           gradients (t > H); 0: the next delayed / eager call is the first outer step */
+  int32_t have_prev;    /* how many generations of delta_prev_local / delta_prev_avg already hold recorded
+                           gradients, 0 .. overlap_steps.  overlap_steps: every delayed / eager call applies
+                           (t > H); 0: the next overlap_steps such calls only record (t <= overlap_steps H) */
   int32_t impl;         /* DILOCO_IMPL_* */
+  int32_t overlap_steps;/* D >= 1: outer steps by which the all-reduce result is delayed.  1 is the paper's
+                           Algorithms 2-3 ("1-outer-step" overlap); 2 is the "two-outer-steps" overlap of
+                           Section 3, for which the paper prints no formula: this library reads it as
+                           line 11 with t-H replaced by t-DH,
+                             g_m = (Delta_m^(t) - Delta_m^(t-DH)) / M + Delta^(t-DH).
+                           At most DILOCO_MAX_OVERLAP. */
 } diloco_config_t;
 
 typedef struct {
   void *theta;             /* [M, stride] fp32 or bf16 per theta_kind: theta_m^(t)                      */
   float *master;           /* [M, stride] fp32, only for DILOCO_THETA_MASTER_BF16, else NULL            */
   float *start;            /* [M, stride] fp32: s_m = theta_m^(t-H)                 (Alg. 1-3 line 7)   */
-  float *delta_prev_local; /* [M, stride] fp32: Delta_m^(t-H); eager only, else may be NULL (Alg. 3 l.11) */
-  float *delta_prev_avg;   /* [stride]    fp32: Delta^(t-H), the all-reduce in flight; delayed and eager,
-                              may be NULL if only the standard step is used         (Alg. 2-3 line 10)  */
+  float *delta_prev_local; /* [D, M, stride] fp32, D = overlap_steps: Delta_m of the last D outer steps, a
+                              ring indexed by (outer-step counter mod D): the step that reads a generation
+                              overwrites it.  Eager only, else may be NULL              (Alg. 3 l.11)    */
+  float *delta_prev_avg;   /* [D, stride] fp32: the means of those steps, i.e. the all-reduces in flight;
+                              delayed and eager, may be NULL if only the standard step is used
+                                                                                    (Alg. 2-3 line 10)  */
   float *outer_mom;        /* [M, stride] fp32: b_m, Nesterov buffer of OuterOpt                        */
   float *adam_m;           /* [M, stride] fp32 first moment;  NULL if diloco_inner_adamw is not used    */
   float *adam_v;           /* [M, stride] fp32 second moment; NULL if diloco_inner_adamw is not used    */
@@ -218,8 +229,10 @@ int diloco_outer_quantized_static(diloco_state_t *state, int32_t variant, int32_
  * The same three steps restricted to parameter indices [offset, offset + len) of every
  * replica (a fragment, as Streaming DiLoCo applies the outer step to parts of the model
  * on different schedules, Section 3).  variant: 0 standard, 1 delayed, 2 eager.  bootstrap
- * != 0 performs the first-outer-step form for this fragment; the state's have_prev flag and
- * outer-step counter are NOT consulted or changed: per-fragment bookkeeping is the caller's.
+ * != 0 performs the first-outer-step form for this fragment; the state's have_prev count is
+ * NOT consulted and neither it nor the outer-step counter is changed: per-fragment
+ * bookkeeping is the caller's (with overlap_steps > 1 the generation used is the one the
+ * outer-step counter currently selects; move it with diloco_state_set_counters).
  * offset must be a multiple of 32 elements (64 if theta is bf16); len >= 1; offset + len <= P.
  */
 int diloco_outer_fragment(diloco_state_t *state, int32_t variant, int32_t bootstrap,

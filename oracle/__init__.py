@@ -104,6 +104,25 @@ def outer_step(variant, *, M, P, stride, eta, mu, theta, start, outer_mom,
         raise ValueError("oracle_outer_step rejected its arguments")
 
 
+def outer_step_overlap(variant, k, have, *, delta_prev_local=None, delta_prev_avg=None, **kw):
+    """Outer step number ``k`` (0-based) of a run whose all-reduce result arrives D outer steps
+    late, D = number of generations in ``delta_prev_avg`` [D, stride] (``delta_prev_local`` is
+    [D, M, stride]).  D = 1 is Algorithms 2-3 as printed.  For D = 2 ("two-outer-steps"
+    overlap, Section 3) the paper prints no formula; the reading taken is line 11 with t-H
+    replaced by t-DH:  g_m = (Delta_m^(t) - Delta_m^(t-DH)) / M + Delta^(t-DH)  (PARITY
+    UNPINNED against the paper: there is nothing printed to pin it to).  The generations are
+    kept in a ring, slot k mod D; the step reads its slot (recorded at step k-D) and then
+    overwrites it.  While fewer than D generations have been recorded (``have`` < D) nothing
+    can have arrived yet and the step only records.  Returns the new ``have``.
+    """
+    D = delta_prev_avg.shape[0]
+    slot = k % D
+    boot = variant != STANDARD and have < D
+    outer_step(variant, bootstrap=boot, delta_prev_avg=delta_prev_avg[slot],
+               delta_prev_local=None if delta_prev_local is None else delta_prev_local[slot], **kw)
+    return min(D, have + 1) if variant != STANDARD else have
+
+
 def eager_gradient(form, *, M, P, stride, theta, start, delta_prev_local, delta_prev_avg=None,
                    master=None, theta_kind=THETA_NATIVE):
     """tilde-Delta_m for all m, without applying it: form 'a' = Alg. 3 line 11, 'b' = the

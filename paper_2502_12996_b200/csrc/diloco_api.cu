@@ -59,7 +59,9 @@ int validate_config(const diloco_config_t *c) {
   if (!std::isfinite(c->outer_lr)) return DILOCO_ERR_INVALID_ARG;
   if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f)) return DILOCO_ERR_INVALID_ARG;
   if (!(c->eps >= 0.f) || !(c->weight_decay >= 0.f)) return DILOCO_ERR_INVALID_ARG;
-  if (c->have_prev != 0 && c->have_prev != 1) return DILOCO_ERR_INVALID_ARG;
+  if (c->overlap_steps < 1) return DILOCO_ERR_INVALID_ARG;
+  if (c->overlap_steps > DILOCO_MAX_OVERLAP) return DILOCO_ERR_UNSUPPORTED;
+  if (c->have_prev < 0 || c->have_prev > c->overlap_steps) return DILOCO_ERR_INVALID_ARG;
   // 128-byte rows for every dtype in use
   if ((c->stride * 4) % 128 != 0) return DILOCO_ERR_MISALIGNED;
   if (c->theta_kind != DILOCO_THETA_F32 && (c->stride * 2) % 128 != 0) return DILOCO_ERR_MISALIGNED;
@@ -140,6 +142,19 @@ int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterA
   }
 }
 
+// Delayed and eager steps consume the gradients recorded overlap_steps outer steps ago: the
+// state keeps that many generations in a ring, slot = outer-step counter mod overlap_steps,
+// and the step that reads a slot overwrites it with the new generation.  Until every slot
+// has been written once (have_prev < overlap_steps) there is nothing to receive yet.
+inline int ring_slot(const diloco_state *st) { return (int)(st->outer_step % st->cfg.overlap_steps); }
+inline bool is_first_steps(const diloco_state *st, int var) {
+  return var != VAR_STANDARD && st->have_prev < st->cfg.overlap_steps;
+}
+inline void advance(diloco_state *st, int var) {
+  if (var != VAR_STANDARD && st->have_prev < st->cfg.overlap_steps) st->have_prev += 1;
+  st->outer_step += 1;
+}
+
 // variant-specific buffer requirements
 int check_variant(const diloco_state *st, int var) {
   if (var < VAR_STANDARD || var > VAR_EAGER) return DILOCO_ERR_INVALID_ARG;
@@ -154,8 +169,9 @@ OuterArgs outer_args(const diloco_state *st, int64_t offset, int64_t len) {
   a.theta = b.theta ? static_cast<char *>(b.theta) + (size_t)offset * theta_elt(st->cfg.theta_kind) : nullptr;
   a.master = b.master ? b.master + offset : nullptr;
   a.start = b.start + offset;
-  a.dpl = b.delta_prev_local ? b.delta_prev_local + offset : nullptr;
-  a.dpa = b.delta_prev_avg ? b.delta_prev_avg + offset : nullptr;
+  const size_t slot = (size_t)ring_slot(st);
+  a.dpl = b.delta_prev_local ? b.delta_prev_local + slot * (size_t)st->cfg.M * (size_t)st->cfg.stride + offset : nullptr;
+  a.dpa = b.delta_prev_avg ? b.delta_prev_avg + slot * (size_t)st->cfg.stride + offset : nullptr;
   a.mom = b.outer_mom + offset;
   a.P = len;
   a.stride = st->cfg.stride;
@@ -266,11 +282,9 @@ int outer_whole(diloco_state *st, int var, void *stream) {
   if (!st) return DILOCO_ERR_INVALID_ARG;
   int rc = check_variant(st, var);
   if (rc != DILOCO_OK) return rc;
-  const bool boot = (var != VAR_STANDARD) && st->have_prev == 0;
-  rc = launch_outer(st, var, boot, 0, st->cfg.P, static_cast<cudaStream_t>(stream));
+  rc = launch_outer(st, var, is_first_steps(st, var), 0, st->cfg.P, static_cast<cudaStream_t>(stream));
   if (rc != DILOCO_OK) return rc;
-  if (var != VAR_STANDARD) st->have_prev = 1;
-  st->outer_step += 1;
+  advance(st, var);
   return DILOCO_OK;
 }
 
@@ -404,12 +418,10 @@ int diloco_outer_quantized(diloco_state_t *st, int32_t variant, int32_t comm_for
     if (exp_bits < 1 || exp_bits > 5 || man_bits < 0 || exp_bits + man_bits > 7) return DILOCO_ERR_INVALID_ARG;
     if (!st->buf.comm_scratch) return DILOCO_ERR_BAD_STATE;
   }
-  const bool boot = (variant != VAR_STANDARD) && st->have_prev == 0;
-  rc = launch_outer_quantized(st, variant, boot, comm_format, exp_bits, man_bits, st->buf.comm_scratch,
-                              static_cast<cudaStream_t>(stream));
+  rc = launch_outer_quantized(st, variant, is_first_steps(st, variant), comm_format, exp_bits, man_bits,
+                              st->buf.comm_scratch, static_cast<cudaStream_t>(stream));
   if (rc != DILOCO_OK) return rc;
-  if (variant != VAR_STANDARD) st->have_prev = 1;
-  st->outer_step += 1;
+  advance(st, variant);
   return DILOCO_OK;
 }
 
@@ -431,13 +443,11 @@ int diloco_outer_quantized_static(diloco_state_t *st, int32_t variant, int32_t c
   rc = static_scratch_for_current_device(dev, &scratch);
   if (rc != DILOCO_OK) return rc;
   if (comm_format == DILOCO_COMM_F32) return outer_whole(st, variant, stream);
-  const bool boot = (variant != VAR_STANDARD) && st->have_prev == 0;
   // launch_outer_quantized zeroes the M words it reduces into before every use
-  rc = launch_outer_quantized(st, variant, boot, comm_format, exp_bits, man_bits, scratch,
+  rc = launch_outer_quantized(st, variant, is_first_steps(st, variant), comm_format, exp_bits, man_bits, scratch,
                               static_cast<cudaStream_t>(stream));
   if (rc != DILOCO_OK) return rc;
-  if (variant != VAR_STANDARD) st->have_prev = 1;
-  st->outer_step += 1;
+  advance(st, variant);
   return DILOCO_OK;
 }
 
@@ -464,8 +474,11 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
   cudaStream_t s_out = static_cast<cudaStream_t>(streams[2]);
   if (s_in == s_k || s_k == s_out || s_in == s_out) return DILOCO_ERR_INVALID_ARG;
   const diloco_buffers_t &d = st->buf;
-  const bool boot = (variant != VAR_STANDARD) && st->have_prev == 0;
+  const bool boot = is_first_steps(st, variant);
   const int tk = st->cfg.theta_kind;
+  const size_t slot = (size_t)ring_slot(st);
+  const size_t slot_rows = slot * (size_t)st->cfg.M * (size_t)st->cfg.stride; // this step's generation
+  const size_t slot_row = slot * (size_t)st->cfg.stride;
   // which buffers the variant reads (in) and writes (out); rows = M, or 1 for delta_prev_avg
   struct Leg { void *dev; void *hst; size_t elt; int rows; bool in, out; };
   const bool master = tk == DILOCO_THETA_MASTER_BF16;
@@ -473,8 +486,12 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
       {d.theta, host->theta, theta_elt(tk), st->cfg.M, !master, !boot},
       {d.master, host->master, 4, st->cfg.M, master, master && !boot},
       {d.start, host->start, 4, st->cfg.M, true, true},
-      {d.delta_prev_local, host->delta_prev_local, 4, st->cfg.M, variant == VAR_EAGER && !boot, variant == VAR_EAGER},
-      {d.delta_prev_avg, host->delta_prev_avg, 4, 1, variant != VAR_STANDARD && !boot, variant != VAR_STANDARD},
+      {d.delta_prev_local ? d.delta_prev_local + slot_rows : nullptr,
+       host->delta_prev_local ? host->delta_prev_local + slot_rows : nullptr, 4, st->cfg.M,
+       variant == VAR_EAGER && !boot, variant == VAR_EAGER},
+      {d.delta_prev_avg ? d.delta_prev_avg + slot_row : nullptr,
+       host->delta_prev_avg ? host->delta_prev_avg + slot_row : nullptr, 4, 1,
+       variant != VAR_STANDARD && !boot, variant != VAR_STANDARD},
       {d.outer_mom, host->outer_mom, 4, st->cfg.M, !boot, !boot},
   };
   for (const Leg &l : legs)
@@ -527,8 +544,7 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
   }
   e = cudaEventRecord(st->last_d2h, s_out);
   if (e != cudaSuccess) return cuda_fail(e);
-  if (variant != VAR_STANDARD) st->have_prev = 1;
-  st->outer_step += 1;
+  advance(st, variant);
   return DILOCO_OK;
 }
 
@@ -541,7 +557,8 @@ int diloco_state_get_counters(const diloco_state_t *st, int64_t *inner_step, int
 }
 
 int diloco_state_set_counters(diloco_state_t *st, int64_t inner_step, int64_t outer_step, int32_t have_prev) {
-  if (!st || inner_step < 0 || outer_step < 0 || (have_prev != 0 && have_prev != 1)) return DILOCO_ERR_INVALID_ARG;
+  if (!st || inner_step < 0 || outer_step < 0 || have_prev < 0 || have_prev > st->cfg.overlap_steps)
+    return DILOCO_ERR_INVALID_ARG;
   st->inner_step = inner_step;
   st->outer_step = outer_step;
   st->have_prev = have_prev;

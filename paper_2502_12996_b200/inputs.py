@@ -97,12 +97,13 @@ def _fill_normal_rows(dst: torch.Tensor, P: int, std: float, gen: torch.Generato
 
 def make_outer_state(M: int, P: int, seed: int, device="cpu", theta_kind: int = THETA_F32,
                      with_adam: bool = False, stride: Optional[int] = None,
-                     gen: Optional[torch.Generator] = None) -> Dict[str, torch.Tensor]:
+                     gen: Optional[torch.Generator] = None, overlap_steps: int = 1) -> Dict[str, torch.Tensor]:
     """Allocate and fill every state buffer of one DiLoCo state on `device`.
 
     Returns a dict with keys theta, master (or None), start, delta_prev_local, delta_prev_avg,
     outer_mom, adam_m, adam_v (or None) and the generator under "gen" for further draws.
-    Padding elements (index >= P) are zero.
+    Padding elements (index >= P) are zero.  With overlap_steps = D > 1 the previous-gradient
+    buffers hold D generations, shaped [D, M, stride] and [D, stride], each drawn like the one.
     """
     stride = padded_stride(P) if stride is None else int(stride)
     dev = torch.device(device)
@@ -122,13 +123,18 @@ def make_outer_state(M: int, P: int, seed: int, device="cpu", theta_kind: int = 
         del noisy
     else:
         theta, master = noisy.to(torch.bfloat16), noisy
-    dpl = torch.zeros((M, stride), **f32)
+    D = int(overlap_steps)
+    dpl = torch.zeros((D * M, stride), **f32)
     _fill_normal_rows(dpl, P, 1e-3, gen)
-    dpa = torch.zeros((stride,), **f32)
-    dpa.copy_(dpl[0])
-    for m in range(1, M):
-        dpa += dpl[m]
+    dpl = dpl.view(D, M, stride)
+    dpa = torch.zeros((D, stride), **f32)
+    for g in range(D):
+        dpa[g].copy_(dpl[g, 0])
+        for m in range(1, M):
+            dpa[g] += dpl[g, m]
     dpa /= float(M)
+    if D == 1:
+        dpl, dpa = dpl[0], dpa[0]
     out = dict(theta=theta, master=master, start=start, delta_prev_local=dpl, delta_prev_avg=dpa,
                outer_mom=torch.zeros((M, stride), **f32), adam_m=None, adam_v=None, gen=gen,
                M=M, P=P, stride=stride, theta_kind=theta_kind)

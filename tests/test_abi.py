@@ -41,7 +41,7 @@ def test_status_strings(lib):
 
 def good_config(**kw):
     c = dict(M=4, H=30, P=1000, stride=1024, outer_lr=0.7, outer_momentum=0.9, beta1=0.9, beta2=0.95, eps=1e-8,
-             weight_decay=0.1, theta_kind=0, grad_kind=0, have_prev=1, impl=0)
+             weight_decay=0.1, theta_kind=0, grad_kind=0, have_prev=1, impl=0, overlap_steps=1)
     c.update(kw)
     return binding.Config(**c)
 
@@ -50,6 +50,7 @@ def good_buffers(**kw):
     b = {k: 0x10000 * (i + 1) for i, k in enumerate(
         ["theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom", "adam_m", "adam_v"])}
     b["device_status"] = None
+    b["comm_scratch"] = None
     b.update(kw)
     return binding.Buffers(**b)
 
@@ -67,13 +68,15 @@ def init(lib, cfg, buf):
 @pytest.mark.parametrize("kw", [dict(M=0), dict(M=-3), dict(P=0), dict(stride=999), dict(theta_kind=3), dict(grad_kind=2),
                                 dict(outer_momentum=1.0), dict(outer_momentum=-0.1), dict(beta1=1.0), dict(beta2=-1.0),
                                 dict(eps=-1e-8), dict(weight_decay=-1.0), dict(have_prev=2), dict(impl=9),
-                                dict(outer_lr=float("nan")), dict(H=-1)])
+                                dict(outer_lr=float("nan")), dict(H=-1), dict(overlap_steps=0), dict(have_prev=-1),
+                                dict(overlap_steps=2, have_prev=3)])
 def test_invalid_config(lib, kw):
     assert init(lib, good_config(**kw), good_buffers()) == binding.ERR_INVALID_ARG
 
 
 def test_unsupported_and_misaligned(lib):
     assert init(lib, good_config(M=65), good_buffers()) == binding.ERR_UNSUPPORTED
+    assert init(lib, good_config(overlap_steps=5), good_buffers()) == binding.ERR_UNSUPPORTED
     assert init(lib, good_config(stride=1000 + 8), good_buffers()) == binding.ERR_MISALIGNED   # 4032 B rows
     assert init(lib, good_config(stride=1024 + 32, theta_kind=1), good_buffers()) == binding.ERR_MISALIGNED  # bf16 rows
     assert init(lib, good_config(), good_buffers(start=0x10008)) == binding.ERR_MISALIGNED

@@ -182,6 +182,63 @@ def test_quantized_argument_checks():
     torch.cuda.synchronize()
 
 
+# ---------------------------------------------------------------- D-outer-steps overlap
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("D,M,P,theta_kind,have", [(2, 4, 150_003, 0, 0), (2, 2, 80_001, 1, 2), (3, 8, 40_002, 0, 1),
+                                                   (4, 16, 20_001, 2, 0), (2, 5, 30_001, 0, 0)])
+def test_overlap_by_D_outer_steps(oracle, variant, D, M, P, theta_kind, have):
+    """All-reduce results consumed D outer steps late (D = 2 is the "two-outer-steps" overlap):
+    D generations of recorded gradients in a ring; runs start with `have` generations seeded."""
+    st = inputs.make_outer_state(M, P, 1900 + D + M, device=DEV, theta_kind=theta_kind, overlap_steps=D)
+    h = host_copy(st)
+    state = binding.State.from_dict(st, have_prev=have, overlap_steps=D)
+    steps = 2 * D + 2
+    for k in range(steps):
+        if k:
+            inputs.inner_phase_standin(st)
+            h["theta"], h["master"] = to_numpy(st["theta"]), to_numpy(st["master"])
+        state.outer(variant)
+        have = oracle.outer_step_overlap(variant, k, have, M=M, P=P, stride=st["stride"], eta=0.7, mu=0.9,
+                                         theta=h["theta"], master=h["master"], start=h["start"],
+                                         outer_mom=h["outer_mom"], delta_prev_local=h["delta_prev_local"],
+                                         delta_prev_avg=h["delta_prev_avg"], theta_kind=theta_kind, nthreads=8)
+        torch.cuda.synchronize()
+        assert_state_equal(st, h, what=f"overlap D={D} {NAMES[variant]} step {k + 1}")
+        assert state.get_counters() == (0, k + 1, have)
+
+
+def test_overlap_with_quantised_wire_and_host_buffers(oracle):
+    """The generation ring is honoured by the quantised call and by the host-buffer call."""
+    D, M, P = 2, 4, 100_003
+    st = inputs.make_outer_state(M, P, 1950, device=DEV, overlap_steps=D)
+    h = host_copy(st)
+    keys = ("theta", "start", "delta_prev_local", "delta_prev_avg", "outer_mom")
+    pinned = {k: st[k].cpu().pin_memory() for k in keys}
+    scratch = torch.zeros(64, dtype=torch.int32, device=DEV)
+    state = binding.State.from_dict(st, overlap_steps=D, comm_scratch=scratch)
+    streams = [torch.cuda.Stream(device=DEV) for _ in range(3)]
+    have = D
+    for k in range(5):
+        if k % 2 == 0:
+            state.outer_quantized(binding.EAGER, binding.COMM_EXMY, 4, 3)
+            torch.cuda.synchronize()
+            for key in keys:
+                pinned[key].copy_(st[key])
+            kw = dict(comm=oracle.COMM_EXMY, exp_bits=4, man_bits=3)
+        else:
+            state.outer_step_host(binding.EAGER, binding.make_buffers(**pinned), streams, 64 * 500)
+            streams[2].synchronize()
+            kw = {}
+        have = oracle.outer_step_overlap(2, k, have, M=M, P=P, stride=st["stride"], eta=0.7, mu=0.9, theta=h["theta"],
+                                         start=h["start"], outer_mom=h["outer_mom"],
+                                         delta_prev_local=h["delta_prev_local"], delta_prev_avg=h["delta_prev_avg"], **kw)
+        assert_state_equal(pinned, h, keys=keys, what=f"overlap mixed step {k + 1}")
+        # next phase: both sides move the replicas the same way
+        inputs.inner_phase_standin(st)
+        h["theta"] = to_numpy(st["theta"])
+        pinned["theta"].copy_(st["theta"])
+
+
 # ---------------------------------------------------------------- inner AdamW
 def run_adamw(oracle, M, P, theta_kind, grad_kind, steps, seed, segments=0):
     st, checks = make(M, P, seed, theta_kind, with_adam=True)
