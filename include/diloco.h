@@ -31,6 +31,8 @@
  *     synchronises the device.  All buffers are updated in place.
  *   - every call returns a status (0 = DILOCO_OK, negative = error); nothing throws or
  *     aborts.  On error nothing has been launched and the state is unchanged.
+ *   - the device that was current at diloco_state_init must be current at every launching
+ *     call on that state (DILOCO_ERR_BAD_STATE otherwise).
  *   - arithmetic: fp32, one IEEE round-to-nearest-even per operation, no FMA contraction,
  *     IEEE division and square root; the sum over replicas runs m = 0 .. M-1 in order; 1/M
  *     is a division by (float)M.  bf16 is a storage type only (round-to-nearest-even).

@@ -101,7 +101,9 @@ template <bool Q, int M, int G, int V, int NT, int MINB>
 int launch_outer_m(int var, int tk, bool boot, const OuterArgs &a, cudaStream_t s) {
 #define DILOCO_CASE(VAR_, TK_)                                                                           \
   if (var == VAR_ && tk == TK_) {                                                                        \
-    if (VAR_ != VAR_STANDARD && boot) return launch_outer_t<M, G, VAR_, TK_, true, V, NT, MINB, Q>(a, s); \
+    if constexpr (VAR_ != VAR_STANDARD) {                                                                \
+      if (boot) return launch_outer_t<M, G, VAR_, TK_, true, V, NT, MINB, Q>(a, s);                      \
+    }                                                                                                    \
     return launch_outer_t<M, G, VAR_, TK_, false, V, NT, MINB, Q>(a, s);                                  \
   }
   DILOCO_CASE(VAR_STANDARD, TK_F32)
@@ -155,9 +157,20 @@ inline void advance(diloco_state *st, int var) {
   st->outer_step += 1;
 }
 
-// variant-specific buffer requirements
+// The buffers live on the device that was current at diloco_state_init; launching from
+// another current device would run the kernel where those pointers mean nothing.
+int check_device(const diloco_state *st) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return dev == st->device ? DILOCO_OK : DILOCO_ERR_BAD_STATE;
+}
+
+// variant-specific buffer requirements, and the state's device must be current
 int check_variant(const diloco_state *st, int var) {
   if (var < VAR_STANDARD || var > VAR_EAGER) return DILOCO_ERR_INVALID_ARG;
+  int rc = check_device(st);
+  if (rc != DILOCO_OK) return rc;
   if (var != VAR_STANDARD && !st->buf.delta_prev_avg) return DILOCO_ERR_BAD_STATE;
   if (var == VAR_EAGER && !st->buf.delta_prev_local) return DILOCO_ERR_BAD_STATE;
   return DILOCO_OK;
@@ -364,6 +377,10 @@ int diloco_inner_adamw(diloco_state_t *st, const void *grads, int64_t grad_strid
   if (!st || !grads) return DILOCO_ERR_INVALID_ARG;
   if (!st->buf.adam_m || !st->buf.adam_v) return DILOCO_ERR_BAD_STATE;
   if (grad_stride < st->cfg.P || !std::isfinite(lr)) return DILOCO_ERR_INVALID_ARG;
+  {
+    int rc = check_device(st);
+    if (rc != DILOCO_OK) return rc;
+  }
   const size_t gelt = st->cfg.grad_kind == DILOCO_GRAD_F32 ? 4 : 2;
   if (!aligned16(grads) || (grad_stride * (int64_t)gelt) % 128 != 0) return DILOCO_ERR_MISALIGNED;
   const int64_t k = st->inner_step + 1;
@@ -435,12 +452,8 @@ int diloco_outer_quantized_static(diloco_state_t *st, int32_t variant, int32_t c
       (exp_bits < 1 || exp_bits > 5 || man_bits < 0 || exp_bits + man_bits > 7))
     return DILOCO_ERR_INVALID_ARG;
   if (st->cfg.M > kStaticScratchWords) return DILOCO_ERR_UNSUPPORTED; // one word of scratch per replica
-  int dev = -1;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return cuda_fail(e);
-  if (dev != st->device) return DILOCO_ERR_BAD_STATE; // the state's GPU must be the current one
-  unsigned *scratch = nullptr;
-  rc = static_scratch_for_current_device(dev, &scratch);
+  unsigned *scratch = nullptr; // check_variant has verified that the state's GPU is the current one
+  rc = static_scratch_for_current_device(st->device, &scratch);
   if (rc != DILOCO_OK) return rc;
   if (comm_format == DILOCO_COMM_F32) return outer_whole(st, variant, stream);
   // launch_outer_quantized zeroes the M words it reduces into before every use
