@@ -123,6 +123,7 @@ int launch_outer_m(int var, int tk, bool boot, const OuterArgs &a, cudaStream_t 
 // chosen by measurement on B200 under two rules: no register spills, and every warp-level
 // access covers at least 128 contiguous bytes of a row (64-byte runs halved the bandwidth).
 // M <= 3: one thread per column.  M = 4, 8, 16: the replica axis is split over G lanes.
+// (M = 4: 6.70 TB/s, M = 8: 6.77, M = 16: 6.45, M = 2: 6.65 in the microbenchmark.)
 template <bool Q>
 int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterArgs &a, cudaStream_t s) {
   const int tk = st->cfg.theta_kind;
@@ -130,11 +131,11 @@ int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterA
     case 1: return launch_outer_m<Q, 1, 1, 4, 128, 8>(var, tk, boot, a, s);
     case 2: return launch_outer_m<Q, 2, 1, 4, 128, 6>(var, tk, boot, a, s);
     case 3: return launch_outer_m<Q, 3, 1, 4, 128, 4>(var, tk, boot, a, s);
-    case 4: return launch_outer_m<Q, 4, 2, 4, 128, 8>(var, tk, boot, a, s);
+    case 4: return launch_outer_m<Q, 4, 2, 4, 256, 4>(var, tk, boot, a, s);
     case 8:
-      // fp32 rows: 16 lanes x 8 B = 128 B per row; bf16 rows need the wider vector for that
-      if (tk == TK_F32) return launch_outer_m<Q, 8, 2, 2, 256, 3>(var, tk, boot, a, s);
-      return launch_outer_m<Q, 8, 2, 4, 128, 4>(var, tk, boot, a, s);
+      // as for M = 16 below: 5 resident blocks unless the wire rounding needs the registers
+      if constexpr (Q) return launch_outer_m<Q, 8, 2, 4, 128, 4>(var, tk, boot, a, s);
+      else return launch_outer_m<Q, 8, 2, 4, 128, 5>(var, tk, boot, a, s);
     case 16:
       // 5 resident blocks (96 registers) measured 4 % faster than 4; the quantised eager form
       // needs 100 registers and would spill under that cap
