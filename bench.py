@@ -40,8 +40,9 @@ FALLBACK_HBM_GBS = 6650.0
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per parameter index for one launch of the
 # dominant kernel, from the captures summarised under profiles/ (None: not captured yet).
 NCU_TRAFFIC_BYTES_PER_PARAM = {
-    ("diloco_outer_eager", 4, 0): 134.37,    # profiles/outer_eager_f32_M4_P35M_cfg1.md
-    ("diloco_inner_adamw", 4, 1): 86.34,     # profiles/inner_adamw_bf16_M4_P35M_cfg2slice.md (35 M slice, scaled by P)
+    ("diloco_outer_eager", 4, 0): 134.38,    # profiles/outer_eager_f32_M4_P35M_cfg1.md
+    ("diloco_inner_adamw", 4, 1): 86.35,     # profiles/inner_adamw_bf16_M4_P35M_cfg2slice.md (35 M slice, scaled by P)
+    ("diloco_outer_eager", 16, 0): 516.2,    # profiles/outer_eager_f32_M16_P15M.md (15 M slice, scaled by P)
 }
 
 
