@@ -211,10 +211,17 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
     if not binding.LIB_PATH.exists():
         build.build_library()
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+    # one rank per GPU; ranks beyond the device count (a gloo dry run on one GPU) share devices
+    backend = os.environ.get("DILOCO_BENCH_BACKEND", "nccl")
+    gpu = local_rank % torch.cuda.device_count()
+    torch.cuda.set_device(gpu)
+    dev = torch.device("cuda", gpu)
+    red_dev = dev if backend == "nccl" else torch.device("cpu")      # where the tiny reductions live
     if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=dev)
+        else:
+            dist.init_process_group(backend)
     w = inputs.WORKLOADS[args.workload]
     P = args.P or w.P                                       # per GPU: weak scaling, every rank the full shape
     if args.strong:                                         # total work fixed: this rank's 64-aligned range
@@ -274,7 +281,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(gpu)
     n0 = binding.launch_count()
     t0 = time.perf_counter()
     rows = [one_step(True) for _ in range(args.steps)]
@@ -288,15 +295,15 @@ def run_ours(args):
     outer_ms = sum(r[1] for r in rows) / len(rows)
     adam_ms = sum(r[2] for r in rows) / len(rows) / max(1, w.H) if phase else None
     if world > 1:
-        t = torch.tensor([step_ms, outer_ms], device=dev, dtype=torch.float64)
+        t = torch.tensor([step_ms, outer_ms], device=red_dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         step_ms, outer_ms = float(t[0]), float(t[1])
-        l = torch.tensor([launches], device=dev)
+        l = torch.tensor([launches], device=red_dev)
         dist.all_reduce(l)
         launches = int(l[0])
     P_job = P * world
     if args.strong:
-        t = torch.tensor([P], device=dev, dtype=torch.int64)
+        t = torch.tensor([P], device=red_dev, dtype=torch.int64)
         if world > 1:
             dist.all_reduce(t)
         P_job = int(t[0])
@@ -309,7 +316,7 @@ def run_ours(args):
     else:
         dom, dom_ms, dom_bpp = f"diloco_outer_{args.variant}", outer_ms, outer_bpp
     achieved = dom_bpp * P / (dom_ms * 1e-3) / 1e9
-    tr = NCU_TRAFFIC_BYTES_PER_PARAM.get((dom, M, w.theta_kind))
+    tr = None if comm[0] else NCU_TRAFFIC_BYTES_PER_PARAM.get((dom, M, w.theta_kind))
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_param": dom_bpp, "traffic": (tr * P if tr else None),
@@ -368,7 +375,7 @@ def run_ours(args):
             per = per[2:]
             e_ms = 1e3 * sum(per) / len(per)
             if world > 1:
-                t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
+                t = torch.tensor([e_ms], device=red_dev, dtype=torch.float64)
                 dist.all_reduce(t, op=dist.ReduceOp.MAX)
                 e_ms = float(t[0])
             def leg_bytes(k):

@@ -405,3 +405,25 @@ def test_non_default_stream(oracle):
     s.synchronize()
     oracle_outer(oracle, 2, h, M, P, st["stride"], 0.7, 0.9, 0)
     assert_state_equal(st, h)
+
+
+# ---------------------------------------------------------------- bench.py, two ranks
+def test_bench_two_ranks_dry_run(tmp_path):
+    """bench.py under torchrun with two ranks (gloo for the barrier and the reductions, both
+    ranks on this one GPU: the ranks never wait on one another's kernels): one JSON line from
+    rank 0, whole-job value = sum over ranks, launches counted on both."""
+    import json, os, subprocess, sys
+    from pathlib import Path
+    root = Path(__file__).resolve().parent.parent
+    env = dict(os.environ, DILOCO_BENCH_BACKEND="gloo")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
+           "127.0.0.1", "--master-port", "29571", str(root / "bench.py"), "--gpus", "2", "--steps", "3", "--warmup", "3",
+           "--P", "2000000", "--no-cpu-baseline", "--no-siblings"]
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env, cwd=str(root))
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["gpu_launches"] == 6 and d["scaling"] == "weak"
+    assert abs(d["value"] - 2 * 2_000_000 / (d["ms_per_step"] * 1e-3)) < 1e-3 * d["value"]
+    assert d["e2e"]["value"] > 0 and d["roofline"]["frac"] > 0
