@@ -340,6 +340,15 @@ def run_ours(args):
             bpp = outer_bytes_per_param(v, M, w.theta_kind)
             kernels[f"outer_{name}"] = {"ms": ms, "GBps": bpp * P / ms / 1e6, "frac": bpp * P / ms / 1e6 / peak,
                                         "params_per_s": P / ms * 1e3}
+        # the worker form: one replica, Delta_m sent / summed Delta received (40 B per index in fp32)
+        if w.theta_kind == 0:
+            sw = binding.State(M=1, P=P, stride=stride, theta=st["theta"][0], start=st["start"][0],
+                               outer_mom=st["outer_mom"][0], delta_prev_local=st["delta_prev_local"].view(-1, stride)[0])
+            send, recv = torch.zeros(stride, device=dev), torch.zeros(stride, device=dev)
+            ms = time_kernel(lambda: sw.worker_outer_apply(binding.EAGER, M, recv, send))
+            kernels["worker_outer_eager"] = {"ms": ms, "GBps": 40 * P / ms / 1e6, "frac": 40 * P / ms / 1e6 / peak,
+                                             "params_per_s": P / ms * 1e3}
+            sw.close(); del send, recv
         if 28 * M * stride < torch.cuda.mem_get_info(dev)[0] * 0.8:
             am = torch.zeros((M, stride), device=dev); av = torch.zeros((M, stride), device=dev)
             g = inputs.make_grads(M, P, stride, st["gen"], dev, 0)

@@ -228,6 +228,39 @@ int diloco_outer_quantized_static(diloco_state_t *state, int32_t variant, int32_
                                   int32_t man_bits, void *cuda_stream);
 
 /*
+ * WORKER FORM of the outer step, for deployments where the M replicas live on M GPUs (one
+ * process per GPU) and line 8's mean is a real all-reduce between them (Section 2.1; the
+ * paper's implementation: an all-reduce without parameter server, Section 3).  The state
+ * holds ONE replica (config M = 1, every [M, stride] buffer is [stride], delta_prev_avg is
+ * not used); the M of the algorithm is world_replicas.  The caller owns the communication:
+ *   delta_send      [>= P] fp32 device buffer the kernel fills with this worker's Delta_m
+ *                   (Alg. 1-3 line 7); all-reduce it with SUM over the workers;
+ *   delta_sum_recv  [>= P] fp32 device buffer holding that element-wise SUM for the outer
+ *                   step whose result is due now; the kernel divides by world_replicas itself,
+ *                   so the arithmetic is Delta = (sum_m Delta_m) / M exactly as in the fused
+ *                   M-replica calls (bit-identical to them when the sum was formed in the
+ *                   order m = 0 .. M-1; for M = 2 every order is that order).
+ * Both 16-byte aligned; nothing else is communicated.
+ *
+ * diloco_worker_outer_send: standard DiLoCo (Algorithm 1) only, lines 7-8: delta_send =
+ *   s - theta, state untouched.  All-reduce it (blocking, line 9), then call
+ *   diloco_worker_outer_apply(variant 0) with the sum: line 10.
+ * diloco_worker_outer_apply, variant 1 (naive delayed) or 2 (eager): one kernel per outer
+ *   step.  It applies OuterOpt with the sum that was sent overlap_steps outer steps ago
+ *   (Algorithm 2 line 11 / Algorithm 3 lines 11-12) and fills delta_send with the new
+ *   Delta_m, whose all-reduce the caller starts asynchronously and lets run during the next
+ *   inner phase.  While have_prev < overlap_steps nothing has arrived yet: delta_sum_recv is
+ *   ignored (may be NULL), the step only records (s <- theta, own Delta_m kept for line 11).
+ *   The worker's own stale gradients live in the state's delta_prev_local ring as usual.
+ * Counters and have_prev advance as in the fused calls.
+ * Errors: INVALID_ARG, MISALIGNED, BAD_STATE (M != 1, delta_prev_local missing for eager,
+ * wrong current device), CUDA.
+ */
+int diloco_worker_outer_send(diloco_state_t *state, float *delta_send, void *cuda_stream);
+int diloco_worker_outer_apply(diloco_state_t *state, int32_t variant, int32_t world_replicas,
+                              const float *delta_sum_recv, float *delta_send, void *cuda_stream);
+
+/*
  * The same three steps restricted to parameter indices [offset, offset + len) of every
  * replica (a fragment, as Streaming DiLoCo applies the outer step to parts of the model
  * on different schedules, Section 3).  variant: 0 standard, 1 delayed, 2 eager.  bootstrap

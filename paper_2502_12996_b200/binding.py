@@ -60,6 +60,8 @@ SYMBOLS = {
     "diloco_outer_eager": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_outer_quantized": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
     "diloco_outer_quantized_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
+    "diloco_worker_outer_send": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_worker_outer_apply": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_outer_fragment": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
     "diloco_outer_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Buffers), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int64]),
     "diloco_state_get_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)]),
@@ -186,6 +188,15 @@ class State:
         """diloco_outer_quantized with the scratch inside the library (no comm_scratch needed)."""
         _check(load_library().diloco_outer_quantized_static(self._handle, variant, comm_format, exp_bits, man_bits,
                                                             _stream_ptr(stream)), "diloco_outer_quantized_static")
+
+    def worker_outer_send(self, delta_send, stream=None) -> None:
+        _check(load_library().diloco_worker_outer_send(self._handle, _ptr(delta_send), _stream_ptr(stream)),
+               "diloco_worker_outer_send")
+
+    def worker_outer_apply(self, variant, world_replicas, delta_sum_recv, delta_send, stream=None) -> None:
+        _check(load_library().diloco_worker_outer_apply(self._handle, variant, world_replicas, _ptr(delta_sum_recv),
+                                                        _ptr(delta_send), _stream_ptr(stream)),
+               "diloco_worker_outer_apply")
 
     def outer_fragment(self, variant, bootstrap, offset, length, stream=None) -> None:
         _check(load_library().diloco_outer_fragment(self._handle, variant, int(bool(bootstrap)), offset, length,

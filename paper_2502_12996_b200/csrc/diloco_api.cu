@@ -14,6 +14,7 @@
 
 #include "diloco_bulk.cuh"
 #include "diloco_kernels.cuh"
+#include "diloco_worker.cuh"
 
 using namespace diloco;
 
@@ -317,6 +318,45 @@ int launch_adamw_t(const diloco_state *st, const AdamArgs &a, cudaStream_t s) {
   return DILOCO_OK;
 }
 
+template <int MODE, int VAR, int TK>
+int launch_worker_t(const WorkerArgs &a, cudaStream_t s) {
+  constexpr int V = 4, NT = 256;
+  long long blocks = (a.P / V + NT - 1) / NT;
+  if (blocks < 1) blocks = 1; // the last block also handles the P % V tail
+  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
+  worker_outer_kernel<MODE, VAR, TK, V, NT><<<(unsigned)blocks, NT, 0, s>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1);
+  return DILOCO_OK;
+}
+
+template <int MODE, int VAR>
+int launch_worker(int tk, const WorkerArgs &a, cudaStream_t s) {
+  switch (tk) {
+    case TK_F32: return launch_worker_t<MODE, VAR, TK_F32>(a, s);
+    case TK_BF16: return launch_worker_t<MODE, VAR, TK_BF16>(a, s);
+    default: return launch_worker_t<MODE, VAR, TK_MASTER_BF16>(a, s);
+  }
+}
+
+WorkerArgs worker_args(const diloco_state *st, int32_t world_replicas, const float *recv, float *send) {
+  WorkerArgs a;
+  const diloco_buffers_t &b = st->buf;
+  a.theta = b.theta;
+  a.master = b.master;
+  a.start = b.start;
+  a.dpl = b.delta_prev_local ? b.delta_prev_local + (size_t)ring_slot(st) * (size_t)st->cfg.stride : nullptr;
+  a.mom = b.outer_mom;
+  a.recv = recv;
+  a.send = send;
+  a.P = st->cfg.P;
+  a.eta = st->cfg.outer_lr;
+  a.mu = st->cfg.outer_momentum;
+  a.fM = (float)world_replicas;
+  return a;
+}
+
 // ---- per-device address of the scratch inside the library image ----------------------------
 constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
@@ -460,6 +500,41 @@ int diloco_outer_quantized_static(diloco_state_t *st, int32_t variant, int32_t c
   // launch_outer_quantized zeroes the M words it reduces into before every use
   rc = launch_outer_quantized(st, variant, is_first_steps(st, variant), comm_format, exp_bits, man_bits, scratch,
                               static_cast<cudaStream_t>(stream));
+  if (rc != DILOCO_OK) return rc;
+  advance(st, variant);
+  return DILOCO_OK;
+}
+
+int diloco_worker_outer_send(diloco_state_t *st, float *delta_send, void *stream) {
+  if (!st || !delta_send) return DILOCO_ERR_INVALID_ARG;
+  if (st->cfg.M != 1) return DILOCO_ERR_BAD_STATE;
+  if (!aligned16(delta_send)) return DILOCO_ERR_MISALIGNED;
+  int rc = check_device(st);
+  if (rc != DILOCO_OK) return rc;
+  WorkerArgs a = worker_args(st, 1, nullptr, delta_send);
+  return launch_worker<WMODE_SEND_ONLY, VAR_STANDARD>(st->cfg.theta_kind, a, static_cast<cudaStream_t>(stream));
+}
+
+int diloco_worker_outer_apply(diloco_state_t *st, int32_t variant, int32_t world_replicas, const float *delta_sum_recv,
+                              float *delta_send, void *stream) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  if (variant < VAR_STANDARD || variant > VAR_EAGER) return DILOCO_ERR_INVALID_ARG;
+  if (world_replicas < 1 || world_replicas > (1 << 24)) return DILOCO_ERR_INVALID_ARG; // exact as a float
+  if (st->cfg.M != 1) return DILOCO_ERR_BAD_STATE;
+  if (variant == VAR_EAGER && !st->buf.delta_prev_local) return DILOCO_ERR_BAD_STATE;
+  const bool first = is_first_steps(st, variant);
+  if (variant != VAR_STANDARD && !delta_send) return DILOCO_ERR_INVALID_ARG;
+  if (!first && !delta_sum_recv) return DILOCO_ERR_INVALID_ARG;
+  if ((delta_send && !aligned16(delta_send)) || (delta_sum_recv && !aligned16(delta_sum_recv))) return DILOCO_ERR_MISALIGNED;
+  int rc = check_device(st);
+  if (rc != DILOCO_OK) return rc;
+  WorkerArgs a = worker_args(st, world_replicas, delta_sum_recv, delta_send);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int tk = st->cfg.theta_kind;
+  if (variant == VAR_STANDARD) rc = launch_worker<WMODE_APPLY, VAR_STANDARD>(tk, a, s);
+  else if (variant == VAR_DELAYED) rc = first ? launch_worker<WMODE_RECORD, VAR_DELAYED>(tk, a, s)
+                                              : launch_worker<WMODE_APPLY_SEND, VAR_DELAYED>(tk, a, s);
+  else rc = first ? launch_worker<WMODE_RECORD, VAR_EAGER>(tk, a, s) : launch_worker<WMODE_APPLY_SEND, VAR_EAGER>(tk, a, s);
   if (rc != DILOCO_OK) return rc;
   advance(st, variant);
   return DILOCO_OK;
