@@ -37,12 +37,17 @@
  *     2^(X-1)-1, subnormals, every code a finite number (no inf/NaN codes),
  *     round to nearest with ties to the even code, saturating; each replica's
  *     vector is scaled so that its largest magnitude maps to the format's
- *     largest value (one fp32 scale per replica per outer step).
+ *     largest value (one fp32 scale per replica per outer step).  PARITY
+ *     UNPINNED against the paper for the EXMY layout and scaling (nothing is
+ *     printed to pin them to); the rounding itself is pinned by brute force
+ *     over every code, the E2M1 value table and a library's float8 casts.
  *
  * Parity pins: every function here is pinned by tests/test_oracle_*.py
  * (hand-worked dyadic example, exact rational brute force, closed forms,
- * torch.optim library routines, invariants); nothing is "parity unpinned"
- * except the readings above themselves, which the paper cannot settle.
+ * torch.optim library routines, invariants).  "Parity unpinned" applies only
+ * to readings that fill gaps the paper leaves open: the EXMY wire format
+ * above, and overlaps of more than one outer step (the ring logic in
+ * __init__.py: outer_step_overlap), for which the paper prints no formula.
  *
  * Layout: every [M, stride] buffer is replica-major, element (m, i) at
  * m*stride + i, only i < P is touched.

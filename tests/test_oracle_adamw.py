@@ -46,22 +46,23 @@ def test_matches_torch_adamw(oracle, dtype, tol):
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float64])
 def test_hand_computed_dyadic_steps(oracle, dtype):
-    """theta0 = 1, g = 1/2, lr = 1/4, wd = 1/2, beta = (1/2, 3/4), eps = 0.
-    k=1: m = 1/4, mhat = 1/2; v = 1/16, vhat = 1/4, sqrt = 1/2; theta = 1 - (1 + 1/2)/4 = 0.625
-    k=2: m = 3/8, mhat = 1/2; v = 7/64, vhat = 1/4;          theta = 0.625 - (1 + 0.3125)/4 = 0.296875
-    (constant gradient: mhat = g and vhat = g^2 at every step).  All values exact in fp32."""
-    hp = dict(lr=0.25, beta1=0.5, beta2=0.75, eps=0.0, wd=0.5)
-    theta = np.full((1, 4), 1.0, dtype)
-    g = np.full((1, 4), 0.5, dtype)
+    """The hand-worked steps of tests/golden/adamw_worked_example.txt (derivation in the file);
+    all values exact in fp32."""
+    from pathlib import Path
+    g = {}
+    for line in (Path(__file__).parent / "golden" / "adamw_worked_example.txt").read_text().splitlines():
+        if line.strip() and not line.startswith("#"):
+            key, val = line.split(":")
+            g[key.strip()] = float(val)
+    hp = dict(lr=g["lr"], beta1=g["beta1"], beta2=g["beta2"], eps=g["eps"], wd=g["wd"])
+    theta = np.full((1, 4), g["theta0"], dtype)
+    grad = np.full((1, 4), g["g"], dtype)
     am, av = np.zeros((1, 4), dtype), np.zeros((1, 4), dtype)
-    run(oracle, theta, [g], am, av, k0=1, hp=hp)
-    np.testing.assert_array_equal(theta, 0.625)
-    np.testing.assert_array_equal(am, 0.25)
-    np.testing.assert_array_equal(av, 0.0625)
-    run(oracle, theta, [g], am, av, k0=2, hp=hp)
-    np.testing.assert_array_equal(theta, 0.296875)
-    np.testing.assert_array_equal(am, 0.375)
-    np.testing.assert_array_equal(av, 0.109375)
+    for k in (1, 2):
+        run(oracle, theta, [grad], am, av, k0=k, hp=hp)
+        np.testing.assert_array_equal(theta, g[f"theta_{k}"])
+        np.testing.assert_array_equal(am, g[f"m_{k}"])
+        np.testing.assert_array_equal(av, g[f"v_{k}"])
 
 
 def test_zero_gradient_is_pure_decay(oracle):
