@@ -121,6 +121,16 @@ class ClockSampler:
                 "samples": len(mhz)}
 
 
+def cpu_model() -> str:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
@@ -192,7 +202,8 @@ def run_reference(args):
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "variant": "eager", "M": w.M, "P": P, "theta": ["f32", "bf16", "f32 master + bf16 copy"][w.theta_kind]},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                             "cpu_model": cpu_model()},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0,
             "note": "the paper ships no code: the reference arm is the CPU oracle (plain C, -O2, no FMA) on the host cores"}
@@ -293,6 +304,8 @@ def run_ours(args):
         dist.barrier()
     step_ms = sum(r[0] for r in rows) / len(rows)
     outer_ms = sum(r[1] for r in rows) / len(rows)
+    outer_sorted = sorted(r[1] for r in rows)
+    outer_median, outer_min = outer_sorted[len(outer_sorted) // 2], outer_sorted[0]
     adam_ms = sum(r[2] for r in rows) / len(rows) / max(1, w.H) if phase else None
     if world > 1:
         t = torch.tensor([step_ms, outer_ms], device=red_dev, dtype=torch.float64)
@@ -320,7 +333,7 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_param": dom_bpp, "traffic": (tr * P if tr else None),
-                "kernel_ms": dom_ms}
+                "kernel_ms": dom_ms, "outer_ms_median": outer_median, "outer_ms_min": outer_min}
 
     # --- extra: the sibling kernels at the same shape (outer-only workloads, rank 0's GPU)
     kernels = {}
@@ -413,7 +426,7 @@ def run_ours(args):
         time_oracle_eager(h, M, Ps, s_stride, w.theta_kind, w.outer_lr, w.outer_momentum, cores, 0, 1)
         tm = time_oracle_eager(h, M, Ps, s_stride, w.theta_kind, w.outer_lr, w.outer_momentum, cores, 8.0)
         t1c = time_oracle_eager(h, M, Ps, s_stride, w.theta_kind, w.outer_lr, w.outer_momentum, 1, 4.0)
-        cpu = {"value": Ps / (sum(tm) / len(tm)), "unit": UNIT, "cores": cores, "kind": "oracle",
+        cpu = {"value": Ps / (sum(tm) / len(tm)), "unit": UNIT, "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
                "sample": f"eager outer step on M={M}, P={Ps} of {P} (all replicas, drawn on the host with the same recipe), "
                          f"{len(tm)} steps with {cores} OpenMP threads",
                "single_thread_value": Ps / (sum(t1c) / len(t1c))}

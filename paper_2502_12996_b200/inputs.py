@@ -19,7 +19,7 @@ Draw order is fixed: s0, theta noise m = 0..M-1, dpl m = 0..M-1, then per-step d
 """
 from __future__ import annotations
 
-from dataclasses import dataclass, field
+from dataclasses import dataclass
 from typing import Dict, List, Optional
 
 import torch
@@ -81,10 +81,6 @@ def generator(seed: int, device) -> torch.Generator:
     g = torch.Generator(device=device)
     g.manual_seed(int(seed))
     return g
-
-
-def _theta_torch_dtype(theta_kind: int):
-    return torch.float32 if theta_kind == THETA_F32 else torch.bfloat16
 
 
 def _fill_normal_rows(dst: torch.Tensor, P: int, std: float, gen: torch.Generator, chunk: int = 1 << 26):
