@@ -129,8 +129,10 @@ typedef struct {
 typedef struct diloco_state diloco_state_t; /* opaque, host memory, owned by the library */
 
 /*
- * Create a state handle: validates config and buffers (ranges, alignment), records the
- * current device and its SM count.  *out is set only on success.  Launches nothing.
+ * Create a state handle: validates config and buffers (ranges, alignment, and that every
+ * buffer pointer is device or managed memory of the current device: a host pointer is
+ * rejected here rather than faulting in a kernel later; sizes cannot be checked), records
+ * the current device and its SM count.  *out is set only on success.  Launches nothing.
  * Errors: INVALID_ARG, MISALIGNED, UNSUPPORTED, CUDA (no usable device).
  */
 int diloco_state_init(const diloco_config_t *config, const diloco_buffers_t *buffers, diloco_state_t **out);

@@ -69,6 +69,20 @@ int validate_config(const diloco_config_t *c) {
   return DILOCO_OK;
 }
 
+// A pointer the kernels will dereference must be device (or managed) memory of `device`;
+// a host pointer here would otherwise surface as an illegal-address fault inside a kernel.
+int check_device_pointer(const void *p, int device) {
+  cudaPointerAttributes at;
+  cudaError_t e = cudaPointerGetAttributes(&at, p);
+  if (e != cudaSuccess) {
+    cudaGetLastError(); // clear the sticky-less error state of the query
+    return DILOCO_ERR_INVALID_ARG;
+  }
+  if (at.type == cudaMemoryTypeManaged) return DILOCO_OK;
+  if (at.type != cudaMemoryTypeDevice || at.device != device) return DILOCO_ERR_INVALID_ARG;
+  return DILOCO_OK;
+}
+
 int validate_buffers(const diloco_config_t *c, const diloco_buffers_t *b) {
   if (!b) return DILOCO_ERR_INVALID_ARG;
   if (!b->theta || !b->start || !b->outer_mom) return DILOCO_ERR_INVALID_ARG;
@@ -392,6 +406,13 @@ int diloco_state_init(const diloco_config_t *config, const diloco_buffers_t *buf
   if (e != cudaSuccess) return cuda_fail(e);
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return cuda_fail(e);
+  {
+    const void *all[] = {buffers->theta, buffers->master, buffers->start, buffers->delta_prev_local,
+                         buffers->delta_prev_avg, buffers->outer_mom, buffers->adam_m, buffers->adam_v,
+                         buffers->device_status, buffers->comm_scratch};
+    for (const void *p : all)
+      if (p && check_device_pointer(p, dev) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
+  }
   diloco_state *st = new (std::nothrow) diloco_state();
   if (!st) return DILOCO_ERR_INVALID_ARG;
   st->cfg = *config;
@@ -424,6 +445,7 @@ int diloco_inner_adamw(diloco_state_t *st, const void *grads, int64_t grad_strid
   }
   const size_t gelt = st->cfg.grad_kind == DILOCO_GRAD_F32 ? 4 : 2;
   if (!aligned16(grads) || (grad_stride * (int64_t)gelt) % 128 != 0) return DILOCO_ERR_MISALIGNED;
+  if (check_device_pointer(grads, st->device) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
   const int64_t k = st->inner_step + 1;
   AdamArgs a;
   a.theta = st->buf.theta;
@@ -511,6 +533,7 @@ int diloco_worker_outer_send(diloco_state_t *st, float *delta_send, void *stream
   if (!aligned16(delta_send)) return DILOCO_ERR_MISALIGNED;
   int rc = check_device(st);
   if (rc != DILOCO_OK) return rc;
+  if (check_device_pointer(delta_send, st->device) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
   WorkerArgs a = worker_args(st, 1, nullptr, delta_send);
   return launch_worker<WMODE_SEND_ONLY, VAR_STANDARD>(st->cfg.theta_kind, a, static_cast<cudaStream_t>(stream));
 }
@@ -528,6 +551,8 @@ int diloco_worker_outer_apply(diloco_state_t *st, int32_t variant, int32_t world
   if ((delta_send && !aligned16(delta_send)) || (delta_sum_recv && !aligned16(delta_sum_recv))) return DILOCO_ERR_MISALIGNED;
   int rc = check_device(st);
   if (rc != DILOCO_OK) return rc;
+  if (delta_send && check_device_pointer(delta_send, st->device) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
+  if (!first && check_device_pointer(delta_sum_recv, st->device) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
   WorkerArgs a = worker_args(st, world_replicas, delta_sum_recv, delta_send);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int tk = st->cfg.theta_kind;

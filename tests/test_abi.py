@@ -102,12 +102,13 @@ def test_null_arguments(lib):
 
 
 def test_valid_arguments_reach_the_device_query(lib):
-    """With valid arguments the only thing left is the device query: OK on a GPU machine, a CUDA
-    error (never a crash, never a silent CPU path) on a box without one."""
+    """With well-formed arguments the next thing is the device: a CUDA error (never a crash,
+    never a silent CPU path) on a box without one; on a GPU machine these made-up addresses are
+    not device memory and are rejected before any kernel could touch them."""
     import torch
     rc = init(lib, good_config(), good_buffers())
     if torch.cuda.is_available():
-        assert rc == 0
+        assert rc == binding.ERR_INVALID_ARG
     else:
         assert rc == binding.ERR_CUDA and binding.last_cuda_error() != 0
 

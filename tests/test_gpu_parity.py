@@ -382,6 +382,27 @@ def test_host_buffer_entry_point(oracle, variant, theta_kind):
     state.close()
 
 
+def test_host_pointers_are_rejected_not_dereferenced():
+    """A host tensor where a device buffer belongs: INVALID_ARG at init (or at the call, for
+    per-call buffers), never a kernel fault."""
+    st, _ = make(2, 1000, 1450, 0, with_adam=True, guards=False)
+    bad = dict(st)
+    bad["start"] = st["start"].cpu()
+    with pytest.raises(binding.DilocoError) as e:
+        binding.State.from_dict(bad)
+    assert e.value.status == binding.ERR_INVALID_ARG
+    bad["start"] = st["start"].cpu().pin_memory()
+    with pytest.raises(binding.DilocoError) as e:
+        binding.State.from_dict(bad)
+    assert e.value.status == binding.ERR_INVALID_ARG
+    state = binding.State.from_dict(st)
+    with pytest.raises(binding.DilocoError) as e:
+        state.inner_adamw(torch.zeros((2, st["stride"])), 1e-3)            # host gradients
+    assert e.value.status == binding.ERR_INVALID_ARG
+    assert state.get_counters()[0] == 0
+    torch.cuda.synchronize()
+
+
 def test_launch_counter():
     M, P = 2, 1000
     st, _ = make(M, P, 1400, 0, with_adam=True)
