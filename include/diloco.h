@@ -281,7 +281,10 @@ int diloco_outer_fragment(diloco_state_t *state, int32_t variant, int32_t bootst
  * dtypes as `state`'s device buffers, which serve as the staging area) to the device,
  * runs the step, and copies every buffer it writes back, chunked along P so that
  * copies and kernels of different chunks overlap on the three streams given.  host: a
- * diloco_buffers_t whose pointers are HOST pointers (pinned memory for full copy speed);
+ * diloco_buffers_t whose pointers are HOST pointers (pinned memory for full copy speed); a
+ * NULL entry means that buffer is resident on the device and is neither copied in nor out
+ * (e.g. only theta travels and the optimiser state stays on the GPU); theta or master must
+ * be given;
  * streams: three distinct cudaStream_t cast to void* (h2d, compute, d2h); chunk: elements
  * per chunk, a multiple of 64.  Returns after enqueueing; the caller synchronises streams[2].
  * Advances have_prev / outer-step counter like the device forms.

@@ -609,7 +609,8 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
       {d.outer_mom, host->outer_mom, 4, st->cfg.M, !boot, !boot},
   };
   for (const Leg &l : legs)
-    if ((l.in || l.out) && (!l.dev || !l.hst)) return DILOCO_ERR_INVALID_ARG;
+    if ((l.in || l.out) && !l.dev) return DILOCO_ERR_INVALID_ARG;
+  if (!host->theta && !host->master) return DILOCO_ERR_INVALID_ARG; // something must come from the host
   const int64_t P = st->cfg.P;
   const size_t nchunks = (size_t)((P + chunk - 1) / chunk);
   cudaError_t e;
@@ -632,7 +633,7 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
     const int64_t off = (int64_t)c * chunk;
     const int64_t len = (off + chunk <= P) ? chunk : (P - off);
     for (const Leg &l : legs) {
-      if (!l.in) continue;
+      if (!l.in || !l.hst) continue; // a NULL host pointer: that buffer is resident on the device
       e = cudaMemcpy2DAsync(static_cast<char *>(l.dev) + (size_t)off * l.elt, row * l.elt,
                             static_cast<const char *>(l.hst) + (size_t)off * l.elt, row * l.elt,
                             (size_t)len * l.elt, (size_t)l.rows, cudaMemcpyHostToDevice, s_in);
@@ -649,7 +650,7 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
     e = cudaStreamWaitEvent(s_out, st->events[2 * c + 1], 0);
     if (e != cudaSuccess) return cuda_fail(e);
     for (const Leg &l : legs) {
-      if (!l.out) continue;
+      if (!l.out || !l.hst) continue;
       e = cudaMemcpy2DAsync(static_cast<char *>(l.hst) + (size_t)off * l.elt, row * l.elt,
                             static_cast<const char *>(l.dev) + (size_t)off * l.elt, row * l.elt,
                             (size_t)len * l.elt, (size_t)l.rows, cudaMemcpyDeviceToHost, s_out);

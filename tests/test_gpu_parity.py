@@ -403,6 +403,24 @@ def test_host_pointers_are_rejected_not_dereferenced():
     torch.cuda.synchronize()
 
 
+def test_host_entry_with_resident_optimizer_state(oracle):
+    """NULL host pointers keep those buffers on the device: only theta crosses the bus."""
+    M, P = 4, 200_003
+    st, _ = make(M, P, 1350, 0, guards=False)
+    h = host_copy(st)
+    theta_host = st["theta"].cpu().pin_memory()
+    st["theta"][:, :P] = -7.0                                    # the device copy must come from the host
+    state = binding.State.from_dict(st)
+    streams = [torch.cuda.Stream(device=DEV) for _ in range(3)]
+    state.outer_step_host(binding.EAGER, binding.make_buffers(theta=theta_host), streams, 64 * 700)
+    streams[2].synchronize()
+    oracle_outer(oracle, 2, h, M, P, st["stride"], 0.7, 0.9, 0)
+    assert_state_equal(dict(st, theta=theta_host), h, what="host path, theta only")
+    assert_state_equal(st, h, what="host path, device copy")
+    with pytest.raises(binding.DilocoError):
+        state.outer_step_host(binding.EAGER, binding.make_buffers(start=theta_host), streams, 64)
+
+
 def test_launch_counter():
     M, P = 2, 1000
     st, _ = make(M, P, 1400, 0, with_adam=True)
