@@ -156,6 +156,9 @@ int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterA
       // needs 100 registers and would spill under that cap
       if constexpr (Q) return launch_outer_m<Q, 16, 4, 4, 128, 4>(var, tk, boot, a, s);
       else return launch_outer_m<Q, 16, 4, 4, 128, 5>(var, tk, boot, a, s);
+    case 32: // 8 replicas per lane; the wire rounding needs 2 blocks' worth of registers
+      if constexpr (Q) return launch_outer_m<Q, 32, 4, 4, 128, 2>(var, tk, boot, a, s);
+      else return launch_outer_m<Q, 32, 4, 4, 128, 3>(var, tk, boot, a, s);
     default: return launch_outer_m<Q, 0, 1, 4, 128, 4>(var, tk, boot, a, s);
   }
 }

@@ -62,7 +62,7 @@ def run_outer_steps(oracle, variant, M, P, theta_kind, steps, seed, have_prev=1,
 
 @pytest.mark.parametrize("variant", [0, 1, 2])
 @pytest.mark.parametrize("M,P", [(1, 70_001), (2, (1 << 20) + 3), (3, 100_003), (4, 300_007), (5, 50_001),
-                                 (8, 200_005), (16, 150_001), (64, 5_003)])
+                                 (8, 200_005), (16, 150_001), (32, 30_001), (64, 5_003)])
 def test_outer_fp32(oracle, variant, M, P):
     run_outer_steps(oracle, variant, M, P, 0, steps=3, seed=100 + M)
 
@@ -139,7 +139,7 @@ FORMATS = {"bf16": (binding.COMM_BF16, 0, 0), "e4m3": (binding.COMM_EXMY, 4, 3),
 @pytest.mark.parametrize("fmt", list(FORMATS))
 @pytest.mark.parametrize("variant", [0, 1, 2])
 @pytest.mark.parametrize("M,P,theta_kind", [(2, 100_003, 0), (4, 300_001, 0), (4, 70_001, 1), (8, 50_002, 2),
-                                            (16, 40_001, 0), (5, 20_003, 0), (1, 9_999, 0)])
+                                            (16, 40_001, 0), (32, 10_001, 1), (5, 20_003, 0), (1, 9_999, 0)])
 def test_quantized_communication(oracle, fmt, variant, M, P, theta_kind):
     """The all-reduce operand rounded to bf16 / scaled EXMY: per-replica maxima reduced on the
     device, same scale, same rounding (ties included), same bits as the oracle; first call is
