@@ -241,6 +241,15 @@ def run_ours(args):
     variant = {"standard": 0, "delayed": 1, "eager": 2}[args.variant]
     M = w.M
     phase = w.H > 0 and not args.outer_only
+    th = {0: 4, 1: 2, 2: 6}[w.theta_kind]
+    need = M * P * (th + 12 + (8 + (2 if w.grad_kind else 4) if phase else 0)) + 4 * P + M * P * 4 + (512 << 20)
+    free = torch.cuda.mem_get_info(dev)[0]
+    if need > free:                                         # report, never run the device out of memory
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "unit": UNIT, "value": None, "n_gpus": world,
+                              "config": {"workload": args.workload},
+                              "skipped": f"needs {need / 2**30:.1f} GiB of device memory, {free / 2**30:.1f} GiB free"}))
+        return 0
     st = inputs.make_outer_state(M, P, w.seed + 1000 * rank, device=dev, theta_kind=w.theta_kind, with_adam=phase)
     stride = st["stride"]
     state = binding.State.from_dict(st, H=w.H, outer_lr=w.outer_lr, outer_momentum=w.outer_momentum, beta1=w.beta1,
@@ -465,6 +474,39 @@ def run_ours(args):
     return 0
 
 
+def report(args):
+    """One bench process per workload (so that each starts from an empty device), all kernels
+    of all five configurations as a table on stderr; the JSON lines go to stdout."""
+    from paper_2502_12996_b200 import inputs
+    rows = []
+    for name, w in inputs.WORKLOADS.items():
+        runs = [["--workload", name, "--steps", str(max(3, args.steps if w.P < 2e8 else 5))]]
+        if w.H:
+            runs = [runs[0] + ["--steps", "3"], runs[0] + ["--outer-only"]]
+        for extra in runs:
+            cmd = [sys.executable, str(ROOT / "bench.py"), "--no-e2e", "--no-cpu-baseline"] + extra
+            out = subprocess.run(cmd, capture_output=True, text=True)
+            line = [l for l in out.stdout.splitlines() if l.startswith("{")]
+            if out.returncode != 0 or not line:
+                rows.append((name, "failed", out.stderr[-200:]))
+                continue
+            print(line[-1])
+            d = json.loads(line[-1])
+            if d.get("skipped"):
+                rows.append((name, "skipped", d["skipped"]))
+                continue
+            r = d["roofline"]
+            rows.append((name, d["config"]["step"], f"M={d['config']['M']} P={d['config']['P_per_gpu']:,} {d['config']['theta']}",
+                         r["kernel"], f"{r['kernel_ms']:.3f} ms", f"{r['achieved']:.0f} GB/s", f"{r['frac']:.3f} {r['peak_kind']}",
+                         f"{r['frac_of_nominal_8000']:.3f} of nominal", f"{d['value']:.3e} params/s",
+                         f"sm {d['clocks']['sm_mhz']} MHz {','.join(d['clocks']['reasons'])}"))
+            for k, v in (d.get("kernels") or {}).items():
+                rows.append((name, "", "", k, f"{v['ms']:.3f} ms", f"{v['GBps']:.0f} GB/s", f"{v['frac']:.3f}", "", f"{v['params_per_s']:.3e} params/s", ""))
+    for r in rows:
+        print(" | ".join(str(x) for x in r), file=sys.stderr)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -483,9 +525,13 @@ def main():
     ap.add_argument("--no-e2e", dest="e2e", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--no-siblings", dest="siblings", action="store_false")
+    ap.add_argument("--report", action="store_true",
+                    help="run every workload (one process each) and print a table of all kernels to stderr")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.report:
+        return report(args)
     return run_reference(args) if args.impl == "reference" else run_ours(args)
 
 
