@@ -29,13 +29,16 @@ class Worker:
 
     def __init__(self, tensors: Dict[str, torch.Tensor], *, P: int, stride: int, world_replicas: int,
                  variant: int = binding.EAGER, overlap_steps: int = 1, have_prev: int = 0,
-                 initial_sums: Optional[List[torch.Tensor]] = None, process_group=None, **hyper):
+                 initial_sums: Optional[List[torch.Tensor]] = None, process_group=None,
+                 state_factory=binding.State, **hyper):
         self.variant, self.D, self.M = variant, int(overlap_steps), int(world_replicas)
         self.group = process_group
         self.have = int(have_prev)
         self.k = 0
         dev = tensors["start"].device
-        self.state = binding.State(M=1, P=P, stride=stride, theta=tensors["theta"], master=tensors.get("master"),
+        # state_factory exists so that the plumbing below can be exercised without a GPU
+        # (a stand-in with the same worker_outer_send / worker_outer_apply / inner_adamw methods)
+        self.state = state_factory(M=1, P=P, stride=stride, theta=tensors["theta"], master=tensors.get("master"),
                                    start=tensors["start"], outer_mom=tensors["outer_mom"],
                                    delta_prev_local=tensors.get("delta_prev_local"), adam_m=tensors.get("adam_m"),
                                    adam_v=tensors.get("adam_v"), have_prev=self.have, overlap_steps=self.D, **hyper)
