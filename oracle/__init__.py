@@ -180,6 +180,35 @@ def exmy_max(exp_bits: int, man_bits: int) -> float:
     return float(fn(exp_bits, man_bits))
 
 
+def wire_encode(d: np.ndarray, exp_bits: int, man_bits: int):
+    """One worker's quantised outer gradient as wire bytes: (payload uint8 array, amax)."""
+    sfx, creal = _prec(d)
+    P = d.shape[0]
+    packed = exp_bits + man_bits + 1 <= 4
+    payload = np.zeros((P + 1) // 2 if packed else P, dtype=np.uint8)
+    amax = np.zeros(1, dtype=d.dtype)
+    fn = getattr(lib(), f"oracle_wire_encode_{sfx}")
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
+    if fn(P, _ptr(np.ascontiguousarray(d)), exp_bits, man_bits, _ptr(payload), _ptr(amax)) != 0:
+        raise ValueError("oracle_wire_encode rejected its arguments")
+    return payload, amax[0]
+
+
+def wire_decode_sum(payloads: np.ndarray, amaxes: np.ndarray, P: int, exp_bits: int, man_bits: int) -> np.ndarray:
+    """Ordered sum over workers of the dequantised payload rows ([M, row bytes] uint8)."""
+    sfx, creal = _prec(amaxes)
+    M = payloads.shape[0]
+    out = np.zeros(P, dtype=amaxes.dtype)
+    fn = getattr(lib(), f"oracle_wire_decode_sum_{sfx}")
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_int, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                   ctypes.c_int, ctypes.c_void_p]
+    if fn(M, P, payloads.strides[0], _ptr(payloads), _ptr(amaxes), exp_bits, man_bits, _ptr(out)) != 0:
+        raise ValueError("oracle_wire_decode_sum rejected its arguments")
+    return out
+
+
 def f32_to_bf16(x: float) -> int:
     fn = lib().oracle_f32_to_bf16_f32
     fn.restype = ctypes.c_uint16

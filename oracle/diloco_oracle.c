@@ -292,6 +292,68 @@ double FN(oracle_exmy_round)(double y, int X, int Y) { return exmy_round(y, X, Y
 double FN(oracle_exmy_max)(int X, int Y) { return exmy_max(X, Y); }
 
 /*
+ * Wire format of one worker's quantised outer gradient (the bytes an EXMY all-gather would
+ * carry; a reading, like EXMY itself: the paper prints none).  Each element is the code
+ * sign << (X+Y) | exponent field << Y | mantissa of R(d / scale), scale = amax / max(EXMY)
+ * (1 if amax = 0), amax = max |d|.  Codes of at most 4 bits are packed two per byte
+ * (element 2j in bits 0-3, element 2j+1 in bits 4-7), wider codes take one byte each.
+ */
+static int wire_packed(int X, int Y) { return X + Y + 1 <= 4; }
+
+int FN(oracle_wire_encode)(int64_t P, const REAL *d, int X, int Y, uint8_t *payload, REAL *amax_out)
+{
+    if (P < 0 || X < 1 || X > 5 || Y < 0 || X + Y > 7) return -1;
+    REAL amax = (REAL)0;
+    for (int64_t i = 0; i < P; ++i) {
+        REAL ab = d[i] < 0 ? -d[i] : d[i];
+        if (ab > amax) amax = ab;
+    }
+    REAL scale = amax > (REAL)0 ? amax / (REAL)exmy_max(X, Y) : (REAL)1;
+    const int packed = wire_packed(X, Y);
+    if (packed) memset(payload, 0, (size_t)((P + 1) / 2));
+    for (int64_t i = 0; i < P; ++i) {
+        REAL y = d[i] / scale;
+        double q = exmy_round((double)y, X, Y);
+        int code = exmy_code(fabs(q), X, Y) | ((signbit(q) ? 1 : 0) << (X + Y));
+        if (packed) payload[i / 2] |= (uint8_t)(code << (4 * (i & 1)));
+        else payload[i] = (uint8_t)code;
+    }
+    *amax_out = amax;
+    return 0;
+}
+
+/* value of a code, from the definition of the format */
+static double exmy_decode(int code, int X, int Y)
+{
+    int bias = (1 << (X - 1)) - 1;
+    int sign = (code >> (X + Y)) & 1;
+    int e = (code >> Y) & ((1 << X) - 1);
+    int m = code & ((1 << Y) - 1);
+    double v = e == 0 ? ldexp((double)m, 1 - bias - Y) : ldexp((double)((1 << Y) + m), e - bias - Y);
+    return sign ? -v : v;
+}
+
+/* sum_out[i] = sum over workers m = 0 .. M-1, in order, of scale_m * value(code_m[i]) */
+int FN(oracle_wire_decode_sum)(int M, int64_t P, int64_t payload_stride, const uint8_t *payloads,
+                               const REAL *amaxes, int X, int Y, REAL *sum_out)
+{
+    if (M < 1 || P < 0 || X < 1 || X > 5 || Y < 0 || X + Y > 7) return -1;
+    const int packed = wire_packed(X, Y);
+    for (int64_t i = 0; i < P; ++i) {
+        REAL acc = (REAL)0;
+        for (int m = 0; m < M; ++m) {
+            const uint8_t *row = payloads + (size_t)m * (size_t)payload_stride;
+            int code = packed ? (row[i / 2] >> (4 * (i & 1))) & 15 : row[i];
+            REAL scale = amaxes[m] > (REAL)0 ? amaxes[m] / (REAL)exmy_max(X, Y) : (REAL)1;
+            REAL w = (REAL)exmy_decode(code, X, Y) * scale;
+            acc = (m == 0) ? w : acc + w;
+        }
+        sum_out[i] = acc;
+    }
+    return 0;
+}
+
+/*
  * The eager outer gradient in the paper's second, equivalent form (Section
  * 2.3 prose): tilde Delta_m = (1/M) (Delta_m^(t) + sum_{m' != m} Delta_{m'}^(t-H)).
  * A real worker cannot evaluate it (it needs every stale local gradient);

@@ -218,3 +218,48 @@ def test_bad_formats_rejected(oracle):
     for X, Y in ((0, 3), (6, 1), (4, 4), (2, -1)):
         with pytest.raises(ValueError):
             run(oracle, 2, st, comm=oracle.COMM_EXMY, exp_bits=X, man_bits=Y)
+
+
+# ---------------------------------------------------------------- wire bytes
+@pytest.mark.parametrize("X,Y", [(4, 3), (5, 2), (2, 1), (3, 0), (3, 2)])
+def test_wire_bytes_against_brute_force_codes(oracle, X, Y):
+    """The payload is the code sign|exponent|mantissa of the rounded, scaled element; 4-bit
+    codes two per byte, low nibble first.  Codes come from the enumerated value table."""
+    rng = np.random.default_rng(20 + X)
+    P = 1001
+    d = rng.normal(0, 1e-3, P).astype(np.float32)
+    d[7] = 0.0
+    payload, amax = oracle.wire_encode(d, X, Y)
+    table = all_values(X, Y)
+    assert amax == np.abs(d).max()
+    scale = np.float32(amax) / np.float32(table[-1][0])
+    codes = []
+    for v in (d / scale).astype(np.float32):
+        a = abs(float(v))
+        val, code = min(table, key=lambda vc: (abs(vc[0] - a), vc[1] & 1))
+        codes.append(code | ((1 if np.signbit(v) else 0) << (X + Y)))
+    codes = np.array(codes, dtype=np.uint8)
+    if X + Y + 1 <= 4:
+        padded = np.concatenate([codes, np.zeros(P % 2, np.uint8)])
+        want = padded[0::2] | (padded[1::2] << 4)
+    else:
+        want = codes
+    np.testing.assert_array_equal(payload, want)
+
+
+@pytest.mark.parametrize("X,Y", [(4, 3), (2, 1), (3, 0)])
+def test_wire_round_trip_is_the_quantised_mean_of_the_step(oracle, X, Y):
+    """Decoding the workers' payloads and summing them in order gives exactly M times the mean
+    that the fused quantised step records."""
+    rng = np.random.default_rng(30 + X)
+    M, P = 4, 777
+    st = state(rng, M, P)
+    d = st["start"] - st["theta"]
+    rows, amaxes = [], []
+    for m in range(M):
+        p, a = oracle.wire_encode(d[m], X, Y)
+        rows.append(p)
+        amaxes.append(a)
+    total = oracle.wire_decode_sum(np.stack(rows), np.array(amaxes, np.float32), P, X, Y)
+    run(oracle, 2, st, comm=oracle.COMM_EXMY, exp_bits=X, man_bits=Y)
+    np.testing.assert_array_equal(total / np.float32(M), st["delta_prev_avg"])
