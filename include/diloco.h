@@ -263,6 +263,37 @@ int diloco_worker_outer_apply(diloco_state_t *state, int32_t variant, int32_t wo
                               const float *delta_sum_recv, float *delta_send, void *cuda_stream);
 
 /*
+ * WORKER FORM WITH A QUANTISED WIRE (Section 3, "Quantized Communication", between real
+ * workers): what a worker sends is its Delta_m as EXMY codes plus one fp32 word, its
+ * max |Delta_m|; the workers exchange these with an ALL-GATHER (a sum of codes means nothing)
+ * and each forms the mean itself,
+ *     Delta = ( sum over m = 0 .. M-1, in order, of scale_m * value(code_m) ) / M,
+ *     scale_m = amax_m / (largest value of the format), or 1 if amax_m = 0,
+ * which is line 8 of diloco_outer_quantized exactly, for any M.  Format as there
+ * (1 <= exp_bits <= 5, exp_bits + man_bits <= 7).  Wire layout: code of an element =
+ * sign << (exp_bits + man_bits) | exponent field << man_bits | mantissa; codes of at most
+ * 4 bits are packed two per byte (element 2j in bits 0-3, element 2j+1 in bits 4-7), wider
+ * codes take one byte each: diloco_wire_payload_bytes(P, ...) bytes per worker, i.e. a quarter
+ * or an eighth of the fp32 gradient.
+ *
+ * diloco_worker_quantized_send: standard DiLoCo, lines 7-8: payload_send and amax_send from
+ *   this worker's Delta_m, state untouched (two kernels: the maximum, then the codes).
+ * diloco_worker_quantized_apply: as diloco_worker_outer_apply.  payloads_recv [world_replicas,
+ *   payload_stride bytes] and amaxes_recv [world_replicas] are the gathered payloads and
+ *   maxima, in worker order, of the outer step whose result is due (ignored while have_prev <
+ *   overlap_steps); for variants 1 and 2 the call also fills payload_send / amax_send with the
+ *   new Delta_m for the gather that runs during the next inner phase.  world_replicas <= 64.
+ * All four buffers: device memory, 4-byte aligned; payload_stride a multiple of 4.
+ */
+int64_t diloco_wire_payload_bytes(int64_t P, int32_t exp_bits, int32_t man_bits);
+int diloco_worker_quantized_send(diloco_state_t *state, int32_t exp_bits, int32_t man_bits, uint8_t *payload_send,
+                                 uint32_t *amax_send, void *cuda_stream);
+int diloco_worker_quantized_apply(diloco_state_t *state, int32_t variant, int32_t world_replicas, int32_t exp_bits,
+                                  int32_t man_bits, const uint8_t *payloads_recv, int64_t payload_stride,
+                                  const uint32_t *amaxes_recv, uint8_t *payload_send, uint32_t *amax_send,
+                                  void *cuda_stream);
+
+/*
  * The same three steps restricted to parameter indices [offset, offset + len) of every
  * replica (a fragment, as Streaming DiLoCo applies the outer step to parts of the model
  * on different schedules, Section 3).  variant: 0 standard, 1 delayed, 2 eager.  bootstrap

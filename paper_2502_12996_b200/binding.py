@@ -62,6 +62,9 @@ SYMBOLS = {
     "diloco_outer_quantized_static": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
     "diloco_worker_outer_send": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_worker_outer_apply": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_wire_payload_bytes": (ctypes.c_int64, [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32]),
+    "diloco_worker_quantized_send": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_worker_quantized_apply": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_outer_fragment": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
     "diloco_outer_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Buffers), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int64]),
     "diloco_state_get_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)]),
@@ -100,6 +103,13 @@ def last_cuda_error() -> int:
 
 def launch_count() -> int:
     return int(load_library().diloco_launch_count())
+
+
+def wire_payload_bytes(P: int, exp_bits: int, man_bits: int) -> int:
+    n = int(load_library().diloco_wire_payload_bytes(P, exp_bits, man_bits))
+    if n < 0:
+        raise DilocoError(n, "diloco_wire_payload_bytes")
+    return n
 
 
 def _check(status: int, where: str) -> None:
@@ -197,6 +207,18 @@ class State:
         _check(load_library().diloco_worker_outer_apply(self._handle, variant, world_replicas, _ptr(delta_sum_recv),
                                                         _ptr(delta_send), _stream_ptr(stream)),
                "diloco_worker_outer_apply")
+
+    def worker_quantized_send(self, exp_bits, man_bits, payload_send, amax_send, stream=None) -> None:
+        _check(load_library().diloco_worker_quantized_send(self._handle, exp_bits, man_bits, _ptr(payload_send),
+                                                           _ptr(amax_send), _stream_ptr(stream)),
+               "diloco_worker_quantized_send")
+
+    def worker_quantized_apply(self, variant, world_replicas, exp_bits, man_bits, payloads_recv, amaxes_recv,
+                               payload_send, amax_send, stream=None) -> None:
+        stride = 0 if payloads_recv is None else payloads_recv.stride(0) * payloads_recv.element_size()
+        _check(load_library().diloco_worker_quantized_apply(
+            self._handle, variant, world_replicas, exp_bits, man_bits, _ptr(payloads_recv), stride, _ptr(amaxes_recv),
+            _ptr(payload_send), _ptr(amax_send), _stream_ptr(stream)), "diloco_worker_quantized_apply")
 
     def outer_fragment(self, variant, bootstrap, offset, length, stream=None) -> None:
         _check(load_library().diloco_outer_fragment(self._handle, variant, int(bool(bootstrap)), offset, length,

@@ -374,6 +374,60 @@ WorkerArgs worker_args(const diloco_state *st, int32_t world_replicas, const flo
   return a;
 }
 
+template <int MODE, int VAR, int TK>
+int launch_worker_q_t(const WorkerQArgs &q, cudaStream_t s) {
+  constexpr int NT = 256;
+  long long blocks = (q.w.P / 4 + NT - 1) / NT;
+  if (blocks < 1) blocks = 1; // the last block also handles the P % 4 tail
+  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
+  worker_quantized_kernel<MODE, VAR, TK, NT><<<(unsigned)blocks, NT, 0, s>>>(q);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1);
+  return DILOCO_OK;
+}
+
+template <int MODE, int VAR>
+int launch_worker_q(int tk, const WorkerQArgs &q, cudaStream_t s) {
+  switch (tk) {
+    case TK_F32: return launch_worker_q_t<MODE, VAR, TK_F32>(q, s);
+    case TK_BF16: return launch_worker_q_t<MODE, VAR, TK_BF16>(q, s);
+    default: return launch_worker_q_t<MODE, VAR, TK_MASTER_BF16>(q, s);
+  }
+}
+
+bool valid_exmy(int X, int Y) { return X >= 1 && X <= 5 && Y >= 0 && X + Y <= 7; }
+
+WorkerQArgs worker_q_args(const diloco_state *st, int world, int X, int Y) {
+  WorkerQArgs q;
+  q.w = worker_args(st, world, nullptr, nullptr);
+  q.precv = nullptr;
+  q.amax_recv = nullptr;
+  q.pstride = 0;
+  q.psend = nullptr;
+  q.amax_send = nullptr;
+  q.world = world;
+  q.man_bits = Y;
+  q.bias = (1 << (X - 1)) - 1;
+  q.emin = 1 - q.bias;
+  q.code_bits = X + Y;
+  q.fmt_max = std::ldexp(2.0f - std::ldexp(1.0f, -Y), (1 << X) - 1 - q.bias);
+  q.packed = (X + Y + 1 <= 4) ? 1 : 0;
+  return q;
+}
+
+// max |Delta_m| of this worker's replica into *amax (zeroed first), on stream s
+int launch_worker_amax(diloco_state *st, unsigned *amax, cudaStream_t s) {
+  cudaError_t e = cudaMemsetAsync(amax, 0, sizeof(unsigned), s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  OuterArgs a = outer_args(st, 0, st->cfg.P);
+  switch (st->cfg.theta_kind) {
+    case TK_F32: return launch_amax_t<TK_F32>(st, a, amax, s);
+    case TK_BF16: return launch_amax_t<TK_BF16>(st, a, amax, s);
+    default: return launch_amax_t<TK_MASTER_BF16>(st, a, amax, s);
+  }
+}
+
 // ---- per-device address of the scratch inside the library image ----------------------------
 constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
@@ -563,6 +617,77 @@ int diloco_worker_outer_apply(diloco_state_t *st, int32_t variant, int32_t world
   else if (variant == VAR_DELAYED) rc = first ? launch_worker<WMODE_RECORD, VAR_DELAYED>(tk, a, s)
                                               : launch_worker<WMODE_APPLY_SEND, VAR_DELAYED>(tk, a, s);
   else rc = first ? launch_worker<WMODE_RECORD, VAR_EAGER>(tk, a, s) : launch_worker<WMODE_APPLY_SEND, VAR_EAGER>(tk, a, s);
+  if (rc != DILOCO_OK) return rc;
+  advance(st, variant);
+  return DILOCO_OK;
+}
+
+int64_t diloco_wire_payload_bytes(int64_t P, int32_t exp_bits, int32_t man_bits) {
+  if (P < 0 || !valid_exmy(exp_bits, man_bits)) return DILOCO_ERR_INVALID_ARG;
+  return (exp_bits + man_bits + 1 <= 4) ? (P + 1) / 2 : P;
+}
+
+int diloco_worker_quantized_send(diloco_state_t *st, int32_t exp_bits, int32_t man_bits, uint8_t *payload_send,
+                                 uint32_t *amax_send, void *stream) {
+  if (!st || !payload_send || !amax_send || !valid_exmy(exp_bits, man_bits)) return DILOCO_ERR_INVALID_ARG;
+  if (st->cfg.M != 1) return DILOCO_ERR_BAD_STATE;
+  if ((reinterpret_cast<uintptr_t>(payload_send) & 3u) || (reinterpret_cast<uintptr_t>(amax_send) & 3u)) return DILOCO_ERR_MISALIGNED;
+  int rc = check_device(st);
+  if (rc != DILOCO_OK) return rc;
+  if (check_device_pointer(payload_send, st->device) != DILOCO_OK || check_device_pointer(amax_send, st->device) != DILOCO_OK)
+    return DILOCO_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  rc = launch_worker_amax(st, amax_send, s);
+  if (rc != DILOCO_OK) return rc;
+  WorkerQArgs q = worker_q_args(st, 1, exp_bits, man_bits);
+  q.psend = payload_send;
+  q.amax_send = amax_send;
+  return launch_worker_q<WMODE_SEND_ONLY, VAR_STANDARD>(st->cfg.theta_kind, q, s);
+}
+
+int diloco_worker_quantized_apply(diloco_state_t *st, int32_t variant, int32_t world_replicas, int32_t exp_bits,
+                                  int32_t man_bits, const uint8_t *payloads_recv, int64_t payload_stride,
+                                  const uint32_t *amaxes_recv, uint8_t *payload_send, uint32_t *amax_send, void *stream) {
+  if (!st || !valid_exmy(exp_bits, man_bits)) return DILOCO_ERR_INVALID_ARG;
+  if (variant < VAR_STANDARD || variant > VAR_EAGER) return DILOCO_ERR_INVALID_ARG;
+  if (world_replicas < 1) return DILOCO_ERR_INVALID_ARG;
+  if (world_replicas > DILOCO_WORKER_MAX_WORLD) return DILOCO_ERR_UNSUPPORTED;
+  if (st->cfg.M != 1) return DILOCO_ERR_BAD_STATE;
+  if (variant == VAR_EAGER && !st->buf.delta_prev_local) return DILOCO_ERR_BAD_STATE;
+  const bool first = is_first_steps(st, variant);
+  const bool sends = variant != VAR_STANDARD;
+  if (sends && (!payload_send || !amax_send)) return DILOCO_ERR_INVALID_ARG;
+  if (!first) {
+    if (!payloads_recv || !amaxes_recv) return DILOCO_ERR_INVALID_ARG;
+    if (payload_stride < diloco_wire_payload_bytes(st->cfg.P, exp_bits, man_bits) || payload_stride % 4 != 0)
+      return DILOCO_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(payloads_recv) & 3u) || (reinterpret_cast<uintptr_t>(amaxes_recv) & 3u)) return DILOCO_ERR_MISALIGNED;
+  }
+  if (sends && ((reinterpret_cast<uintptr_t>(payload_send) & 3u) || (reinterpret_cast<uintptr_t>(amax_send) & 3u))) return DILOCO_ERR_MISALIGNED;
+  int rc = check_device(st);
+  if (rc != DILOCO_OK) return rc;
+  if (!first && (check_device_pointer(payloads_recv, st->device) != DILOCO_OK ||
+                 check_device_pointer(amaxes_recv, st->device) != DILOCO_OK))
+    return DILOCO_ERR_INVALID_ARG;
+  if (sends && (check_device_pointer(payload_send, st->device) != DILOCO_OK ||
+                check_device_pointer(amax_send, st->device) != DILOCO_OK))
+    return DILOCO_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (sends) {
+    rc = launch_worker_amax(st, amax_send, s);
+    if (rc != DILOCO_OK) return rc;
+  }
+  WorkerQArgs q = worker_q_args(st, world_replicas, exp_bits, man_bits);
+  q.precv = payloads_recv;
+  q.amax_recv = amaxes_recv;
+  q.pstride = payload_stride;
+  q.psend = payload_send;
+  q.amax_send = amax_send;
+  const int tk = st->cfg.theta_kind;
+  if (variant == VAR_STANDARD) rc = launch_worker_q<WMODE_APPLY, VAR_STANDARD>(tk, q, s);
+  else if (variant == VAR_DELAYED) rc = first ? launch_worker_q<WMODE_RECORD, VAR_DELAYED>(tk, q, s)
+                                              : launch_worker_q<WMODE_APPLY_SEND, VAR_DELAYED>(tk, q, s);
+  else rc = first ? launch_worker_q<WMODE_RECORD, VAR_EAGER>(tk, q, s) : launch_worker_q<WMODE_APPLY_SEND, VAR_EAGER>(tk, q, s);
   if (rc != DILOCO_OK) return rc;
   advance(st, variant);
   return DILOCO_OK;

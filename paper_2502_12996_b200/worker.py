@@ -30,7 +30,7 @@ class Worker:
     def __init__(self, tensors: Dict[str, torch.Tensor], *, P: int, stride: int, world_replicas: int,
                  variant: int = binding.EAGER, overlap_steps: int = 1, have_prev: int = 0,
                  initial_sums: Optional[List[torch.Tensor]] = None, process_group=None,
-                 state_factory=binding.State, **hyper):
+                 state_factory=binding.State, wire: Optional[tuple] = None, **hyper):
         self.variant, self.D, self.M = variant, int(overlap_steps), int(world_replicas)
         self.group = process_group
         self.have = int(have_prev)
@@ -47,6 +47,17 @@ class Worker:
         # the one being read
         self.ring = [torch.zeros(stride, dtype=torch.float32, device=dev) for _ in range(self.D + 1)]
         self.pending: Dict[int, object] = {}
+        # quantised wire (exp_bits, man_bits): the workers exchange EXMY codes + one fp32 word
+        # by all-gather; slot k keeps what this worker sent and everything it gathered
+        self.wire = wire
+        if wire is not None:
+            if self.have:
+                raise ValueError("a quantised run starts with have_prev = 0")
+            nbytes = (binding.wire_payload_bytes(P, *wire) + 15) // 16 * 16
+            u8, i32 = dict(dtype=torch.uint8, device=dev), dict(dtype=torch.int32, device=dev)
+            self.qring = [dict(send=torch.zeros(nbytes, **u8), amax=torch.zeros(1, **i32),
+                               gathered=torch.zeros((self.M, nbytes), **u8), amaxes=torch.zeros(self.M, **i32))
+                          for _ in range(self.D + 1)]
         if self.have:
             if initial_sums is None or len(initial_sums) != self.have:
                 raise ValueError("have_prev generations need their all-reduced sums")
@@ -59,7 +70,34 @@ class Worker:
     def _all_reduce(self, t: torch.Tensor, async_op: bool):
         return dist.all_reduce(t, op=dist.ReduceOp.SUM, group=self.group, async_op=async_op)
 
+    def _all_gather(self, slot: dict, async_op: bool):
+        works = [dist.all_gather_into_tensor(slot["gathered"].view(-1), slot["send"], group=self.group, async_op=async_op),
+                 dist.all_gather_into_tensor(slot["amaxes"], slot["amax"], group=self.group, async_op=async_op)]
+        return works if async_op else None
+
+    def _outer_step_quantized(self) -> None:
+        k, D, (X, Y) = self.k, self.D, self.wire
+        if self.variant == binding.STANDARD:
+            slot = self.qring[0]
+            self.state.worker_quantized_send(X, Y, slot["send"], slot["amax"])
+            self._all_gather(slot, async_op=False)
+            self.state.worker_quantized_apply(binding.STANDARD, self.M, X, Y, slot["gathered"], slot["amaxes"], None, None)
+        else:
+            mine = self.qring[k % (D + 1)]
+            due = None
+            if self.have >= D:
+                for work in self.pending.pop(k - D, ()):
+                    work.wait()
+                due = self.qring[(k - D) % (D + 1)]
+            self.state.worker_quantized_apply(self.variant, self.M, X, Y, None if due is None else due["gathered"],
+                                              None if due is None else due["amaxes"], mine["send"], mine["amax"])
+            self.pending[k] = self._all_gather(mine, async_op=True)
+            self.have = min(D, self.have + 1)
+        self.k += 1
+
     def outer_step(self) -> None:
+        if self.wire is not None:
+            return self._outer_step_quantized()
         k, D = self.k, self.D
         if self.variant == binding.STANDARD:
             # Algorithm 1: send, block on the all-reduce (line 9), apply
@@ -83,7 +121,8 @@ class Worker:
     def finish(self) -> None:
         """Wait for the all-reduces still in flight (end of training)."""
         for work in self.pending.values():
-            work.wait()
+            for w in (work if isinstance(work, (list, tuple)) else (work,)):
+                w.wait()
         self.pending.clear()
 
     def close(self) -> None:

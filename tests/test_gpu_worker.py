@@ -87,6 +87,65 @@ def test_workers_with_ordered_sum_equal_the_fused_oracle(oracle, variant, M, P, 
         s.close()
 
 
+@pytest.mark.parametrize("fmt", [(4, 3), (2, 1), (3, 0), (5, 2), (3, 2)])
+@pytest.mark.parametrize("variant,M,P,theta_kind,D", [(2, 4, 70_001, 0, 1), (2, 3, 30_002, 1, 2), (1, 2, 20_003, 0, 1),
+                                                      (0, 5, 10_001, 2, 1), (2, 1, 999, 0, 1)])
+def test_quantised_wire_workers_equal_the_fused_quantised_oracle(oracle, fmt, variant, M, P, theta_kind, D):
+    """Each worker sends EXMY codes + its maximum, gathers everyone's, and forms the mean itself:
+    bit-identical to the fused quantised oracle for ANY M (a gather keeps the worker order), and
+    the bytes on the wire equal the oracle's encoding."""
+    X, Y = fmt
+    st = inputs.make_outer_state(M, P, 2300 + M + D, device=DEV, theta_kind=theta_kind, overlap_steps=D)
+    stride = st["stride"]
+    h = host_copy(st)
+    dpl = st["delta_prev_local"].view(D, M, stride)
+    states = [binding.State(M=1, P=P, stride=stride, theta=st["theta"][m], master=row(st["master"], m),
+                            start=st["start"][m], outer_mom=st["outer_mom"][m],
+                            delta_prev_local=dpl[:, m].contiguous() if variant == 2 else None,
+                            theta_kind=theta_kind, have_prev=0, overlap_steps=D) for m in range(M)]
+    nbytes = (binding.wire_payload_bytes(P, X, Y) + 15) // 16 * 16
+    ring = [dict(gathered=torch.zeros((M, nbytes), dtype=torch.uint8, device=DEV),
+                 amaxes=torch.zeros(M, dtype=torch.int32, device=DEV)) for _ in range(D)]
+    h["delta_prev_local"] = h["delta_prev_local"].reshape(D, M, stride)
+    h["delta_prev_avg"] = h["delta_prev_avg"].reshape(D, stride)
+    hv = 0
+    for k in range(2 * D + 2):
+        if k:
+            inputs.inner_phase_standin(st)
+            h["theta"], h["master"] = to_numpy(st["theta"]), to_numpy(st["master"])
+        slot = ring[k % D]
+        new = dict(gathered=torch.zeros_like(slot["gathered"]), amaxes=torch.zeros_like(slot["amaxes"]))
+        d_before = h["start"] - (h["master"] if theta_kind == 2 else
+                                 (h["theta"] if theta_kind == 0 else
+                                  torch.tensor(h["theta"].view(np.int16)).view(torch.bfloat16).float().numpy()))
+        for m in range(M):                                  # "send" phase of every worker
+            if variant == 0:
+                states[m].worker_quantized_send(X, Y, new["gathered"][m], new["amaxes"][m:m + 1])
+            else:
+                states[m].worker_quantized_apply(variant, M, X, Y, slot["gathered"] if hv >= D else None,
+                                                 slot["amaxes"] if hv >= D else None, new["gathered"][m],
+                                                 new["amaxes"][m:m + 1])
+        if variant == 0:
+            for m in range(M):
+                states[m].worker_quantized_apply(0, M, X, Y, new["gathered"], new["amaxes"], None, None)
+        ring[k % D] = new
+        torch.cuda.synchronize()
+        # wire bytes against the oracle's encoder
+        for m in range(M):
+            want, amax = oracle.wire_encode(np.ascontiguousarray(d_before[m, :P]), X, Y)
+            got = new["gathered"][m].cpu().numpy()
+            np.testing.assert_array_equal(got[:len(want)], want)
+            assert new["amaxes"][m].cpu().numpy().view(np.float32) == np.float32(amax)
+        hv = oracle.outer_step_overlap(variant, k, hv, M=M, P=P, stride=stride, eta=0.7, mu=0.9, theta=h["theta"],
+                                       master=h["master"], start=h["start"], outer_mom=h["outer_mom"],
+                                       delta_prev_local=h["delta_prev_local"], delta_prev_avg=h["delta_prev_avg"],
+                                       theta_kind=theta_kind, comm=oracle.COMM_EXMY, exp_bits=X, man_bits=Y)
+        got = dict(theta=st["theta"], master=st["master"], start=st["start"], outer_mom=st["outer_mom"])
+        assert_state_equal(got, h, keys=tuple(got), what=f"quantised wire {fmt} variant {variant} M={M} step {k + 1}")
+    for s_ in states:
+        s_.close()
+
+
 def test_worker_argument_checks():
     st = inputs.make_outer_state(2, 1000, 1, device=DEV)
     two = binding.State.from_dict(st)
@@ -115,7 +174,7 @@ def _free_port():
         return s.getsockname()[1]
 
 
-def _rank_main(rank, world, port, variant, D, P, H, phases, theta_kind, out_dir):
+def _rank_main(rank, world, port, variant, D, P, H, phases, theta_kind, out_dir, wire=None):
     import torch.distributed as dist
     sys.path.insert(0, str(ROOT))
     from paper_2502_12996_b200 import inputs as inp, worker
@@ -130,7 +189,7 @@ def _rank_main(rank, world, port, variant, D, P, H, phases, theta_kind, out_dir)
                 adam_m=st["adam_m"][rank].clone(), adam_v=st["adam_v"][rank].clone(),
                 delta_prev_local=torch.zeros((D, stride), device="cuda:0"))
     w = worker.Worker(mine, P=P, stride=stride, world_replicas=world, variant=variant, overlap_steps=D, have_prev=0,
-                      theta_kind=theta_kind, grad_kind=theta_kind and 1, H=H)
+                      theta_kind=theta_kind, grad_kind=theta_kind and 1, H=H, wire=wire)
     gdt = torch.bfloat16 if theta_kind else torch.float32
     for ph in range(phases):
         for _ in range(H):
@@ -144,12 +203,14 @@ def _rank_main(rank, world, port, variant, D, P, H, phases, theta_kind, out_dir)
     dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("variant,D,theta_kind", [(2, 1, 0), (2, 2, 1), (1, 1, 0), (0, 1, 0)])
-def test_two_worker_processes_with_async_all_reduce(oracle, tmp_path, variant, D, theta_kind):
+@pytest.mark.parametrize("variant,D,theta_kind,wire", [(2, 1, 0, None), (2, 2, 1, None), (1, 1, 0, None), (0, 1, 0, None),
+                                                       (2, 1, 0, (4, 3)), (2, 2, 1, (2, 1)), (0, 1, 0, (3, 0))])
+def test_two_worker_processes_with_async_all_reduce(oracle, tmp_path, variant, D, theta_kind, wire):
     import torch.multiprocessing as mp
     world, P, H, phases = 2, 60_001, 3, 2 * D + 2
-    mp.spawn(_rank_main, args=(world, _free_port(), variant, D, P, H, phases, theta_kind, str(tmp_path)), nprocs=world,
-             join=True)
+    mp.spawn(_rank_main, args=(world, _free_port(), variant, D, P, H, phases, theta_kind, str(tmp_path), wire),
+             nprocs=world, join=True)
+    comm_kw = {} if wire is None else dict(comm=oracle.COMM_EXMY, exp_bits=wire[0], man_bits=wire[1])
     # the same run through the fused oracle
     st = inputs.make_outer_state(world, P, 777, device=DEV, theta_kind=theta_kind, with_adam=True, overlap_steps=D)
     stride = st["stride"]
@@ -168,7 +229,7 @@ def test_two_worker_processes_with_async_all_reduce(oracle, tmp_path, variant, D
         have = oracle.outer_step_overlap(variant, ph, have, M=world, P=P, stride=stride, eta=0.7, mu=0.9,
                                          theta=h["theta"], master=h["master"], start=h["start"], outer_mom=h["outer_mom"],
                                          delta_prev_local=h["delta_prev_local"], delta_prev_avg=h["delta_prev_avg"],
-                                         theta_kind=theta_kind)
+                                         theta_kind=theta_kind, **comm_kw)
     for r in range(world):
         z = np.load(tmp_path / f"rank{r}.npz")
         for key in ("theta", "start", "outer_mom", "adam_m", "adam_v"):
