@@ -10,13 +10,14 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libdiloco.so"
 REPORT = PKG / "ptxas_report.txt"        # registers / spills of every kernel, written by each build
-SOURCES = [CSRC / "diloco_api.cu"]
+OUTER_M = [0, 1, 2, 3, 4, 8, 16, 32]    # replica counts with a translation unit of their own (0 = runtime-M)
+OBJ = PKG / "_obj"
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
     "-fmad=false",                       # no FMA contraction: one rounding per operation
     "-prec-div=true", "-prec-sqrt=true", "-ftz=false",
-    "--cudart", "static", "-shared", "-Xcompiler", "-fPIC",
+    "-Xcompiler", "-fPIC", "-Xptxas", "-v",
 ]
 
 
@@ -28,18 +29,34 @@ def _stale() -> bool:
     return any(d.stat().st_mtime > t for d in deps)
 
 
+def _compile(nvcc: str, src: Path, obj: Path, defines) -> str:
+    cmd = [nvcc] + NVCC_FLAGS + [f"-D{d}" for d in defines] + ["-c", str(src), "-o", str(obj)]
+    res = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+    if res.returncode != 0:
+        print(res.stdout)
+        raise subprocess.CalledProcessError(res.returncode, cmd)
+    return res.stdout
+
+
 def build_library(force: bool = False, verbose: bool = False) -> Path:
+    """Compile the host/ABI unit and one unit per replica count side by side, then link."""
     if not force and not _stale() and REPORT.exists():
         return LIB
+    from concurrent.futures import ThreadPoolExecutor
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    OBJ.mkdir(exist_ok=True)
+    jobs = [(CSRC / "diloco_api.cu", OBJ / "diloco_api.o", [])]
+    jobs += [(CSRC / "diloco_outer_m.cu", OBJ / f"diloco_outer_m{m}.o", [f"DILOCO_M={m}"]) for m in OUTER_M]
+    with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as pool:
+        logs = list(pool.map(lambda j: _compile(nvcc, *j), jobs))
     tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = [nvcc] + NVCC_FLAGS + ["-Xptxas", "-v", "-o", str(tmp)] + [str(s) for s in SOURCES]
-    res = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
-    if verbose or res.returncode != 0:
-        print(res.stdout)
-    if res.returncode != 0:
-        raise subprocess.CalledProcessError(res.returncode, cmd)
-    REPORT.write_text(res.stdout)
+    link = [nvcc, "-shared", "--cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a", "-o", str(tmp)] \
+        + [str(j[1]) for j in jobs]
+    subprocess.check_call(link)
+    report = "\n".join(logs)
+    if verbose:
+        print(report)
+    REPORT.write_text(report)
     os.replace(tmp, LIB)
     return LIB
 

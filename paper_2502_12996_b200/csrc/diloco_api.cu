@@ -14,9 +14,17 @@
 
 #include "diloco_bulk.cuh"
 #include "diloco_kernels.cuh"
+#include "diloco_outer_launch.cuh"
 #include "diloco_worker.cuh"
 
 using namespace diloco;
+
+// launch_outer_shape<M, Q> is instantiated in diloco_outer_m.cu, once per replica count
+#define DILOCO_EXTERN(M_)                                                                                       \
+  extern template int diloco::launch_outer_shape<M_, false>(int, int, bool, const OuterArgs &, cudaStream_t); \
+  extern template int diloco::launch_outer_shape<M_, true>(int, int, bool, const OuterArgs &, cudaStream_t);
+DILOCO_FOR_EACH_M(DILOCO_EXTERN)
+#undef DILOCO_EXTERN
 
 struct diloco_state {
   diloco_config_t cfg;
@@ -36,14 +44,17 @@ constexpr int kStaticScratchWords = DILOCO_MAX_M;
 static __device__ __align__(256) unsigned g_static_scratch[kStaticScratchWords];
 
 namespace {
-
 std::atomic<int64_t> g_launches{0};
 std::atomic<int32_t> g_last_cuda_error{0};
+} // namespace
 
-int cuda_fail(cudaError_t e) {
+int diloco::cuda_fail(cudaError_t e) {
   g_last_cuda_error.store((int32_t)e);
   return DILOCO_ERR_CUDA;
 }
+void diloco::count_launch() { g_launches.fetch_add(1); }
+
+namespace {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -97,69 +108,16 @@ int validate_buffers(const diloco_config_t *c, const diloco_buffers_t *b) {
   return DILOCO_OK;
 }
 
-template <int M, int G, int VAR, int TK, bool BOOT, int V, int NT, int MINB, bool Q>
-int launch_outer_t(const OuterArgs &a, cudaStream_t s) {
-  constexpr int CW = 32 / G;
-  const long long nvec = a.P / V;
-  const long long warps = (nvec + CW - 1) / CW;
-  long long blocks = (warps * 32 + NT - 1) / NT;
-  if (blocks < 1) blocks = 1; // the last block also handles the P % V tail
-  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
-  outer_step_kernel<M, G, VAR, TK, BOOT, V, NT, MINB, Q><<<(unsigned)blocks, NT, 0, s>>>(a);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(e);
-  g_launches.fetch_add(1);
-  return DILOCO_OK;
-}
-
-template <bool Q, int M, int G, int V, int NT, int MINB>
-int launch_outer_m(int var, int tk, bool boot, const OuterArgs &a, cudaStream_t s) {
-#define DILOCO_CASE(VAR_, TK_)                                                                           \
-  if (var == VAR_ && tk == TK_) {                                                                        \
-    if constexpr (VAR_ != VAR_STANDARD) {                                                                \
-      if (boot) return launch_outer_t<M, G, VAR_, TK_, true, V, NT, MINB, Q>(a, s);                      \
-    }                                                                                                    \
-    return launch_outer_t<M, G, VAR_, TK_, false, V, NT, MINB, Q>(a, s);                                  \
-  }
-  DILOCO_CASE(VAR_STANDARD, TK_F32)
-  DILOCO_CASE(VAR_STANDARD, TK_BF16)
-  DILOCO_CASE(VAR_STANDARD, TK_MASTER_BF16)
-  DILOCO_CASE(VAR_DELAYED, TK_F32)
-  DILOCO_CASE(VAR_DELAYED, TK_BF16)
-  DILOCO_CASE(VAR_DELAYED, TK_MASTER_BF16)
-  DILOCO_CASE(VAR_EAGER, TK_F32)
-  DILOCO_CASE(VAR_EAGER, TK_BF16)
-  DILOCO_CASE(VAR_EAGER, TK_MASTER_BF16)
-#undef DILOCO_CASE
-  return DILOCO_ERR_INVALID_ARG;
-}
-
-// Launch shapes per M (lane groups G, vector width V, threads NT, min resident blocks MINB),
-// chosen by measurement on B200 under two rules: no register spills, and every warp-level
-// access covers at least 128 contiguous bytes of a row (64-byte runs halved the bandwidth).
-// M <= 3: one thread per column.  M = 4, 8, 16: the replica axis is split over G lanes.
-// (M = 4: 6.70 TB/s, M = 8: 6.77, M = 16: 6.45, M = 2: 6.65 in the microbenchmark.)
 template <bool Q>
 int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterArgs &a, cudaStream_t s) {
   const int tk = st->cfg.theta_kind;
   switch (st->cfg.M) {
-    case 1: return launch_outer_m<Q, 1, 1, 4, 128, 8>(var, tk, boot, a, s);
-    case 2: return launch_outer_m<Q, 2, 1, 4, 128, 6>(var, tk, boot, a, s);
-    case 3: return launch_outer_m<Q, 3, 1, 4, 128, 4>(var, tk, boot, a, s);
-    case 4: return launch_outer_m<Q, 4, 2, 4, 256, 4>(var, tk, boot, a, s);
-    case 8:
-      // as for M = 16 below: 5 resident blocks unless the wire rounding needs the registers
-      if constexpr (Q) return launch_outer_m<Q, 8, 2, 4, 128, 4>(var, tk, boot, a, s);
-      else return launch_outer_m<Q, 8, 2, 4, 128, 5>(var, tk, boot, a, s);
-    case 16:
-      // 5 resident blocks (96 registers) measured 4 % faster than 4; the quantised eager form
-      // needs 100 registers and would spill under that cap
-      if constexpr (Q) return launch_outer_m<Q, 16, 4, 4, 128, 4>(var, tk, boot, a, s);
-      else return launch_outer_m<Q, 16, 4, 4, 128, 5>(var, tk, boot, a, s);
-    case 32: // 8 replicas per lane; the wire rounding needs 2 blocks' worth of registers
-      if constexpr (Q) return launch_outer_m<Q, 32, 4, 4, 128, 2>(var, tk, boot, a, s);
-      else return launch_outer_m<Q, 32, 4, 4, 128, 3>(var, tk, boot, a, s);
-    default: return launch_outer_m<Q, 0, 1, 4, 128, 4>(var, tk, boot, a, s);
+#define DILOCO_DISPATCH(M_) \
+  case M_: return launch_outer_shape<M_, Q>(var, tk, boot, a, s);
+    DILOCO_DISPATCH(1) DILOCO_DISPATCH(2) DILOCO_DISPATCH(3) DILOCO_DISPATCH(4) DILOCO_DISPATCH(8) DILOCO_DISPATCH(16)
+    DILOCO_DISPATCH(32)
+#undef DILOCO_DISPATCH
+    default: return launch_outer_shape<0, Q>(var, tk, boot, a, s);
   }
 }
 
