@@ -163,8 +163,10 @@ int diloco_outer_standard(diloco_state_t *state, void *cuda_stream);
 /*
  * Outer step with naive delayed outer gradients, Algorithm 2 lines 7-11: as above but
  * OuterOpt consumes delta_prev_avg (the mean formed at the previous outer step), and the new
- * mean replaces it afterwards.  If have_prev == 0 (t = H) nothing is applied: the mean is
- * recorded, s_m <- theta_m, theta and outer_mom are unchanged, have_prev becomes 1.
+ * mean replaces it afterwards.  While have_prev < overlap_steps (t = H with the paper's
+ * overlap of one outer step) nothing is applied: the mean is recorded, s_m <- theta_m, theta
+ * and outer_mom are unchanged, have_prev grows by one.  With overlap_steps = D > 1 the mean
+ * consumed is the one recorded D outer steps ago (generation ring, see diloco_buffers_t).
  * Errors additionally: BAD_STATE (delta_prev_avg missing).
  */
 int diloco_outer_delayed(diloco_state_t *state, void *cuda_stream);
@@ -175,7 +177,8 @@ int diloco_outer_delayed(diloco_state_t *state, void *cuda_stream);
  *     g_m = (Delta_m - delta_prev_local_m) / M + delta_prev_avg          (line 11)
  *     b_m <- mu b_m + g_m;  s_m <- s_m - eta (g_m + mu b_m);  theta_m <- s_m  (line 12)
  *     delta_prev_local_m <- Delta_m;  delta_prev_avg <- Delta.
- * have_prev == 0: first outer step, as for diloco_outer_delayed, also recording Delta_m.
+ * have_prev < overlap_steps: first outer step(s), as for diloco_outer_delayed, also recording
+ * Delta_m; overlap_steps = D > 1: delta_prev_local / delta_prev_avg of D outer steps ago.
  * Errors additionally: BAD_STATE (delta_prev_local or delta_prev_avg missing).
  */
 int diloco_outer_eager(diloco_state_t *state, void *cuda_stream);
