@@ -25,7 +25,9 @@
  *     0 <= i < P <= stride.  Elements with i >= P are padding: never read, never written.
  *     stride * sizeof(element) must be a multiple of 128 bytes for every buffer (so stride
  *     is a multiple of 64 when any buffer is bf16, else of 32), base pointers 16-byte
- *     aligned.  grads use their own stride with the same rule.
+ *     aligned.  grads use their own stride with the same rule.  (Performance, not
+ *     correctness: rows that start on 4 KB boundaries, i.e. a stride that is a multiple of
+ *     1024 elements, measured 1-2 % faster on B200.)
  *   - all kernels are launched asynchronously on the stream the caller passes
  *     (a cudaStream_t cast to void*; NULL = the legacy default stream).  No call
  *     synchronises the device.  All buffers are updated in place.

@@ -31,8 +31,11 @@ BASE_SEED = 12996
 
 
 def padded_stride(P: int) -> int:
-    """Smallest stride >= P whose row is a multiple of 128 bytes for fp32 and for bf16 rows."""
-    return (int(P) + 63) // 64 * 64
+    """Row stride for a vector of P elements: the library needs rows that are multiples of 128
+    bytes (64 elements covers bf16 rows too); rows that start on 4 KB boundaries measured 1-2 %
+    faster on B200 (M = 4, 8), so the stride is rounded up to 1024 elements.  (Coarser
+    alignments, up to 8 MB, were tried at the full benchmark sizes: within run-to-run noise.)"""
+    return (int(P) + 1023) // 1024 * 1024
 
 
 @dataclass
