@@ -75,7 +75,7 @@ def load_peak():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    """nvidia-smi clocks and throttle reasons sampled every 100 ms from the warm-up on; the timed region's own samples are used when there are at least three."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -84,7 +84,7 @@ class ClockSampler:
         self.rows, self.proc = [], None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "200", "-i", str(index)], stdout=subprocess.PIPE,
+                                          "-lms", "100", "-i", str(index)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -95,7 +95,7 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
 
-    def stop(self, t0: float, t1: float):
+    def stop(self, t0: float, t1: float, t_fallback: float = None):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.25)
@@ -104,7 +104,13 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        rows = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.25] or [r for (_, r) in self.rows]
+        rows = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.25]
+        window = "timed region"
+        if len(rows) < 3 and t_fallback is not None:       # under load since the warm-up began
+            rows = [r for (t, r) in self.rows if t_fallback <= t <= t1 + 0.25]
+            window = "warm-up + timed region"
+        if not rows:
+            rows, window = [r for (_, r) in self.rows], "whole run"
         mhz, mx, reasons = [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
@@ -118,7 +124,7 @@ class ClockSampler:
                     reasons.add(n)
         mhz.sort()
         return {"sm_mhz": (mhz[len(mhz) // 2] if mhz else None), "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(mhz)}
+                "samples": len(mhz), "window": window}
 
 
 def cpu_model() -> str:
@@ -296,19 +302,20 @@ def run_ours(args):
         e2.synchronize()
         return e0.elapsed_time(e2), e1.elapsed_time(e2), e0.elapsed_time(e1)
 
+    sampler = ClockSampler(gpu)                            # started before the warm-up: a short timed region
+    t_warm = time.perf_counter()                           # may see too few 100 ms samples of its own
     for _ in range(args.warmup):
         one_step(False)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    sampler = ClockSampler(gpu)
     n0 = binding.launch_count()
     t0 = time.perf_counter()
     rows = [one_step(True) for _ in range(args.steps)]
     torch.cuda.synchronize()
     t1 = time.perf_counter()
     launches = binding.launch_count() - n0
-    clocks = sampler.stop(t0, t1)
+    clocks = sampler.stop(t0, t1, t_warm)
     if world > 1:
         dist.barrier()
     step_ms = sum(r[0] for r in rows) / len(rows)
