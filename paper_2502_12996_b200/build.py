@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libdiloco.so"
 REPORT = PKG / "ptxas_report.txt"        # registers / spills of every kernel, written by each build
-OUTER_M = [0, 1, 2, 3, 4, 8, 16, 32]    # replica counts with a translation unit of their own (0 = runtime-M)
+OUTER_M = [0, 1, 2, 3, 4, 8, 16, 32, 64]    # replica counts with a translation unit of their own (0 = runtime-M)
 OBJ = PKG / "_obj"
 
 NVCC_FLAGS = [
@@ -18,7 +18,7 @@ NVCC_FLAGS = [
     "-fmad=false",                       # no FMA contraction: one rounding per operation
     "-prec-div=true", "-prec-sqrt=true", "-ftz=false",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v",
-]
+] + os.environ.get("DILOCO_EXTRA_NVCC_FLAGS", "").split()
 
 
 def _stale() -> bool:

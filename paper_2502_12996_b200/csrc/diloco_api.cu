@@ -115,7 +115,7 @@ int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterA
 #define DILOCO_DISPATCH(M_) \
   case M_: return launch_outer_shape<M_, Q>(var, tk, boot, a, s);
     DILOCO_DISPATCH(1) DILOCO_DISPATCH(2) DILOCO_DISPATCH(3) DILOCO_DISPATCH(4) DILOCO_DISPATCH(8) DILOCO_DISPATCH(16)
-    DILOCO_DISPATCH(32)
+    DILOCO_DISPATCH(32) DILOCO_DISPATCH(64)
 #undef DILOCO_DISPATCH
     default: return launch_outer_shape<0, Q>(var, tk, boot, a, s);
   }

@@ -477,6 +477,104 @@ __global__ void __launch_bounds__(NT, MINB) outer_step_kernel(const OuterArgs a)
   }
 }
 
+// ---------------------------------------------------------------- outer step, many replicas
+// M = 64 does not fit the lane split: 8 or 16 lanes per column would leave 64- or 32-byte runs
+// per row.  Here the replica axis is split across the WARPS of a block instead: warp w owns
+// replicas 4w .. 4w+3 of 32 columns (32 V-element vectors per row and access), every warp
+// leaves what its replicas send (Delta_m, or its wire rounding) in shared memory, and after
+// one barrier every thread sums all M contributions of its own 4 indices in the order
+// m = 0 .. M-1: the same left-to-right sum as everywhere else.  Block = M/4 warps.
+template <int M, int VAR, int TK, bool BOOT, bool Q, int V, int MINB>
+__global__ void __launch_bounds__(8 * M, MINB) outer_step_cta_kernel(const OuterArgs a) {
+  static_assert(M % 4 == 0 && M >= 8 && M <= 128, "one warp per 4 replicas, at most 32 warps");
+  constexpr int R = 4;
+  __shared__ float sent[M][V][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int m0 = warp * R;
+  const long long nvec = a.P / V;
+  const long long j = (long long)blockIdx.x * 32 + lane;
+  const bool active = j < nvec;
+  const long long i = j * V;
+  float s[R][V], d[R][V], b[R][V], pl[R][V], pa[V], x[R][V], mean[V];
+  if (active) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const long long at = (m0 + r) * a.stride + i;
+      F32Vec<V>::load(a.start + at, s[r]);
+      load_theta<TK, V>(a, at, d[r]);
+      if (!BOOT) {
+        F32Vec<V>::load(a.mom + at, b[r]);
+        if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + at, pl[r]);
+      }
+    }
+    if (!BOOT && VAR != VAR_STANDARD) F32Vec<V>::load(a.dpa + i, pa);
+  } else {
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int e = 0; e < V; ++e) s[r][e] = d[r][e] = 0.f;
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const float scale = Q ? comm_scale(a, m0 + r) : 1.f;
+    float w[V];
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      x[r][e] = d[r][e];
+      d[r][e] = s[r][e] - d[r][e];                                  // Alg. 1-3 line 7
+      w[e] = Q ? comm_round(d[r][e], scale, a) : d[r][e];
+    }
+#pragma unroll
+    for (int e = 0; e < V; ++e) sent[m0 + r][e][lane] = w[e];
+  }
+  __syncthreads();
+  // line 8: Delta = (1/M) sum_m (what replica m sent), m in order
+#pragma unroll 8
+  for (int m = 0; m < M; ++m) {
+#pragma unroll
+    for (int e = 0; e < V; ++e) mean[e] = (m == 0) ? sent[m][e][lane] : mean[e] + sent[m][e][lane];
+  }
+#pragma unroll
+  for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
+  if (active) {
+    if constexpr (BOOT) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const long long at = (m0 + r) * a.stride + i;
+        F32Vec<V>::store(a.start + at, x[r]);
+        if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d[r]);
+      }
+      if (warp == 0) F32Vec<V>::store(a.dpa + i, mean);
+    } else {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const long long at = (m0 + r) * a.stride + i;
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          float g;
+          if (VAR == VAR_STANDARD) g = mean[e];
+          else if (VAR == VAR_DELAYED) g = pa[e];
+          else {
+            float t = d[r][e] - pl[r][e];                            // Alg. 3 line 11
+            t = t / a.fM;
+            g = t + pa[e];
+          }
+          nesterov(g, a.eta, a.mu, b[r][e], s[r][e]);
+        }
+        F32Vec<V>::store(a.mom + at, b[r]);
+        F32Vec<V>::store(a.start + at, s[r]);
+        store_theta<TK, V>(a, at, s[r]);
+        if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d[r]);
+      }
+      if (VAR != VAR_STANDARD && warp == 0) F32Vec<V>::store(a.dpa + i, mean);
+    }
+  }
+  if (blockIdx.x == gridDim.x - 1) { // ragged tail, one index per thread
+    const long long t = nvec * V + threadIdx.x;
+    if (t < a.P) outer_column_rt<VAR, TK, BOOT, 1, Q>(a, t);
+  }
+}
+
 // ---------------------------------------------------------------- inner AdamW
 // U columns of one thread: all loads of all U columns are issued before the first use, so a
 // thread keeps U x (theta, g, m, v) vectors in flight.

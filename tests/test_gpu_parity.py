@@ -69,14 +69,14 @@ def test_outer_fp32(oracle, variant, M, P):
 
 @pytest.mark.parametrize("variant", [0, 1, 2])
 @pytest.mark.parametrize("theta_kind", [1, 2])
-@pytest.mark.parametrize("M,P", [(2, 100_001), (4, 250_003), (7, 20_001), (8, 60_002), (16, 40_003)])
+@pytest.mark.parametrize("M,P", [(2, 100_001), (4, 250_003), (7, 20_001), (8, 60_002), (16, 40_003), (64, 7_003)])
 def test_outer_bf16_storage(oracle, variant, theta_kind, M, P):
     run_outer_steps(oracle, variant, M, P, theta_kind, steps=3, seed=200 + M)
 
 
 @pytest.mark.parametrize("variant", [1, 2])
 @pytest.mark.parametrize("theta_kind", [0, 1, 2])
-@pytest.mark.parametrize("M", [2, 4, 6, 16])
+@pytest.mark.parametrize("M", [2, 4, 6, 16, 64])
 def test_first_outer_step_then_regular(oracle, variant, theta_kind, M):
     """have_prev = 0: the first call records and applies nothing (t = H), later calls apply."""
     run_outer_steps(oracle, variant, M, 33_335, theta_kind, steps=3, seed=300 + M, have_prev=0)
@@ -139,7 +139,7 @@ FORMATS = {"bf16": (binding.COMM_BF16, 0, 0), "e4m3": (binding.COMM_EXMY, 4, 3),
 @pytest.mark.parametrize("fmt", list(FORMATS))
 @pytest.mark.parametrize("variant", [0, 1, 2])
 @pytest.mark.parametrize("M,P,theta_kind", [(2, 100_003, 0), (4, 300_001, 0), (4, 70_001, 1), (8, 50_002, 2),
-                                            (16, 40_001, 0), (32, 10_001, 1), (5, 20_003, 0), (1, 9_999, 0)])
+                                            (16, 40_001, 0), (32, 10_001, 1), (64, 9_001, 2), (5, 20_003, 0), (1, 9_999, 0)])
 def test_quantized_communication(oracle, fmt, variant, M, P, theta_kind):
     """The all-reduce operand rounded to bf16 / scaled EXMY: per-replica maxima reduced on the
     device, same scale, same rounding (ties included), same bits as the oracle; first call is
