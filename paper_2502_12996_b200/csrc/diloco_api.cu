@@ -110,15 +110,18 @@ int validate_buffers(const diloco_config_t *c, const diloco_buffers_t *b) {
 
 template <bool Q>
 int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterArgs &a, cudaStream_t s) {
-  const int tk = st->cfg.theta_kind;
-  switch (st->cfg.M) {
-#define DILOCO_DISPATCH(M_) \
-  case M_: return launch_outer_shape<M_, Q>(var, tk, boot, a, s);
-    DILOCO_DISPATCH(1) DILOCO_DISPATCH(2) DILOCO_DISPATCH(3) DILOCO_DISPATCH(4) DILOCO_DISPATCH(8) DILOCO_DISPATCH(16)
-    DILOCO_DISPATCH(32) DILOCO_DISPATCH(64)
-#undef DILOCO_DISPATCH
-    default: return launch_outer_shape<0, Q>(var, tk, boot, a, s);
+  const int tk = st->cfg.theta_kind, M = st->cfg.M;
+  switch (M) {
+    case 1: return launch_outer_shape<1, Q>(var, tk, boot, a, s);
+    case 2: return launch_outer_shape<2, Q>(var, tk, boot, a, s);
+    case 3: return launch_outer_shape<3, Q>(var, tk, boot, a, s);
+    case 4: return launch_outer_shape<4, Q>(var, tk, boot, a, s);
+    case 8: return launch_outer_shape<8, Q>(var, tk, boot, a, s);
+    default: break;
   }
+  if (M % 4 == 0) return launch_outer_shape<SHAPE_WARP_SPLIT, Q>(var, tk, boot, a, s);       // 12, 16, ..., 64
+  if (M <= 7) return launch_outer_shape<SHAPE_WARP_PER_REPLICA, Q>(var, tk, boot, a, s);     // 5, 6, 7
+  return launch_outer_shape<SHAPE_TWO_SWEEP, Q>(var, tk, boot, a, s);
 }
 
 // Delayed and eager steps consume the gradients recorded overlap_steps outer steps ago: the

@@ -478,17 +478,17 @@ __global__ void __launch_bounds__(NT, MINB) outer_step_kernel(const OuterArgs a)
 }
 
 // ---------------------------------------------------------------- outer step, many replicas
-// M = 64 does not fit the lane split: 8 or 16 lanes per column would leave 64- or 32-byte runs
-// per row.  Here the replica axis is split across the WARPS of a block instead: warp w owns
+// Large M does not fit the lane split: 8 or 16 lanes per column would leave 64- or 32-byte
+// runs per row.  Here the replica axis is split across the WARPS of a block instead: warp w owns
 // replicas 4w .. 4w+3 of 32 columns (32 V-element vectors per row and access), every warp
 // leaves what its replicas send (Delta_m, or its wire rounding) in shared memory, and after
 // one barrier every thread sums all M contributions of its own 4 indices in the order
-// m = 0 .. M-1: the same left-to-right sum as everywhere else.  Block = M/4 warps.
-template <int M, int VAR, int TK, bool BOOT, bool Q, int V, int MINB>
-__global__ void __launch_bounds__(8 * M, MINB) outer_step_cta_kernel(const OuterArgs a) {
-  static_assert(M % 4 == 0 && M >= 8 && M <= 128, "one warp per 4 replicas, at most 32 warps");
-  constexpr int R = 4;
-  __shared__ float sent[M][V][32];
+// m = 0 .. M-1: the same left-to-right sum as everywhere else.  Block = M/4 warps; M is a
+// run-time multiple of 4 (12 .. 64), so one set of kernels serves all of them.
+template <int VAR, int TK, bool BOOT, bool Q, int V>
+__global__ void __launch_bounds__(512, 2) outer_step_cta_kernel(const OuterArgs a) {
+  constexpr int R = 4;                 // a.M is a multiple of 4, at most 64: block = 8 M threads
+  extern __shared__ float sent_dyn[];  // [M][V][32]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int m0 = warp * R;
   const long long nvec = a.P / V;
@@ -525,14 +525,17 @@ __global__ void __launch_bounds__(8 * M, MINB) outer_step_cta_kernel(const Outer
       w[e] = Q ? comm_round(d[r][e], scale, a) : d[r][e];
     }
 #pragma unroll
-    for (int e = 0; e < V; ++e) sent[m0 + r][e][lane] = w[e];
+    for (int e = 0; e < V; ++e) sent_dyn[((m0 + r) * V + e) * 32 + lane] = w[e];
   }
   __syncthreads();
   // line 8: Delta = (1/M) sum_m (what replica m sent), m in order
-#pragma unroll 8
-  for (int m = 0; m < M; ++m) {
+#pragma unroll 4
+  for (int m = 0; m < a.M; ++m) {
 #pragma unroll
-    for (int e = 0; e < V; ++e) mean[e] = (m == 0) ? sent[m][e][lane] : mean[e] + sent[m][e][lane];
+    for (int e = 0; e < V; ++e) {
+      const float w = sent_dyn[(m * V + e) * 32 + lane];
+      mean[e] = (m == 0) ? w : mean[e] + w;
+    }
   }
 #pragma unroll
   for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
@@ -567,6 +570,81 @@ __global__ void __launch_bounds__(8 * M, MINB) outer_step_cta_kernel(const Outer
         if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d[r]);
       }
       if (VAR != VAR_STANDARD && warp == 0) F32Vec<V>::store(a.dpa + i, mean);
+    }
+  }
+  if (blockIdx.x == gridDim.x - 1) { // ragged tail, one index per thread
+    const long long t = nvec * V + threadIdx.x;
+    if (t < a.P) outer_column_rt<VAR, TK, BOOT, 1, Q>(a, t);
+  }
+}
+
+// ---------------------------------------------------------------- outer step, small odd M
+// One warp per replica, M <= 8 chosen at launch (block = 32 M threads, shared memory M x V x 32
+// floats): warp m owns replica m of 32 columns, leaves what it sends in shared memory, and
+// after one barrier every thread forms the ordered sum m = 0 .. M-1 for its own indices.
+// Serves the small replica counts that have no compile-time shape (5, 6, 7); with more warps
+// per block the barrier costs more than it saves (M = 12: 5.0 TB/s, M = 24: 3.4).
+template <int VAR, int TK, bool BOOT, bool Q, int V>
+__global__ void __launch_bounds__(256, 4) outer_step_warp_per_replica_kernel(const OuterArgs a) {
+  extern __shared__ float sent_dyn[]; // [M][V][32]
+  const int lane = threadIdx.x & 31, m = threadIdx.x >> 5;
+  const long long nvec = a.P / V;
+  const long long j = (long long)blockIdx.x * 32 + lane;
+  const bool active = j < nvec;
+  const long long i = j * V, at = m * a.stride + i;
+  float s[V], d[V], b[V], pl[V], pa[V], x[V], mean[V];
+  if (active) {
+    F32Vec<V>::load(a.start + at, s);
+    load_theta<TK, V>(a, at, d);
+    if (!BOOT) {
+      F32Vec<V>::load(a.mom + at, b);
+      if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + at, pl);
+      if (VAR != VAR_STANDARD) F32Vec<V>::load(a.dpa + i, pa);
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < V; ++e) s[e] = d[e] = 0.f;
+  }
+  const float scale = Q ? comm_scale(a, m) : 1.f;
+#pragma unroll
+  for (int e = 0; e < V; ++e) {
+    x[e] = d[e];
+    d[e] = s[e] - d[e];                                             // Alg. 1-3 line 7
+    sent_dyn[(m * V + e) * 32 + lane] = Q ? comm_round(d[e], scale, a) : d[e];
+  }
+  __syncthreads();
+  for (int q = 0; q < a.M; ++q) {                                   // line 8, replica order
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      const float w = sent_dyn[(q * V + e) * 32 + lane];
+      mean[e] = (q == 0) ? w : mean[e] + w;
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
+  if (active) {
+    if constexpr (BOOT) {
+      F32Vec<V>::store(a.start + at, x);
+      if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d);
+      if (m == 0) F32Vec<V>::store(a.dpa + i, mean);
+    } else {
+#pragma unroll
+      for (int e = 0; e < V; ++e) {
+        float g;
+        if (VAR == VAR_STANDARD) g = mean[e];
+        else if (VAR == VAR_DELAYED) g = pa[e];
+        else {
+          float t = d[e] - pl[e];                                    // Alg. 3 line 11
+          t = t / a.fM;
+          g = t + pa[e];
+        }
+        nesterov(g, a.eta, a.mu, b[e], s[e]);
+      }
+      F32Vec<V>::store(a.mom + at, b);
+      F32Vec<V>::store(a.start + at, s);
+      store_theta<TK, V>(a, at, s);
+      if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d);
+      if (VAR != VAR_STANDARD && m == 0) F32Vec<V>::store(a.dpa + i, mean);
     }
   }
   if (blockIdx.x == gridDim.x - 1) { // ragged tail, one index per thread

@@ -62,7 +62,7 @@ def run_outer_steps(oracle, variant, M, P, theta_kind, steps, seed, have_prev=1,
 
 @pytest.mark.parametrize("variant", [0, 1, 2])
 @pytest.mark.parametrize("M,P", [(1, 70_001), (2, (1 << 20) + 3), (3, 100_003), (4, 300_007), (5, 50_001),
-                                 (8, 200_005), (16, 150_001), (32, 30_001), (64, 5_003)])
+                                 (8, 200_005), (12, 40_003), (16, 150_001), (24, 9_001), (32, 30_001), (64, 5_003)])
 def test_outer_fp32(oracle, variant, M, P):
     run_outer_steps(oracle, variant, M, P, 0, steps=3, seed=100 + M)
 
