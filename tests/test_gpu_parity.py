@@ -451,12 +451,15 @@ def test_bench_two_ranks_dry_run(tmp_path):
     """bench.py under torchrun with two ranks (gloo for the barrier and the reductions, both
     ranks on this one GPU: the ranks never wait on one another's kernels): one JSON line from
     rank 0, whole-job value = sum over ranks, launches counted on both."""
-    import json, os, subprocess, sys
+    import json, os, socket, subprocess, sys
     from pathlib import Path
     root = Path(__file__).resolve().parent.parent
     env = dict(os.environ, DILOCO_BENCH_BACKEND="gloo")
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
-           "127.0.0.1", "--master-port", "29571", str(root / "bench.py"), "--gpus", "2", "--steps", "3", "--warmup", "3",
+           "127.0.0.1", "--master-port", str(port), str(root / "bench.py"), "--gpus", "2", "--steps", "3", "--warmup", "3",
            "--P", "2000000", "--no-cpu-baseline", "--no-siblings"]
     out = subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env, cwd=str(root))
     assert out.returncode == 0, out.stderr[-2000:]
