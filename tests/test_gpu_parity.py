@@ -498,3 +498,47 @@ def test_bench_line_has_every_contract_key():
     assert d["e2e"]["h2d_bytes_per_step"] == 3000000 * (4 * 16 + 4) and d["e2e"]["value"] < d["value"]
     for k in ("sm_mhz", "sm_max_mhz", "reasons"):
         assert k in d["clocks"], k
+
+
+# ---------------------------------------------------------------- seeded random sweep
+@pytest.mark.parametrize("case", range(48))
+def test_random_configurations(oracle, case):
+    """Seeded random (M, P, variant, storage, overlap, wire format, seeded generations): every
+    replica count from 1 to 64 lands on one of the kernel forms (per-thread, lane split, warp
+    split, warp per replica, two sweeps), and every combination must equal the oracle bit for
+    bit over several outer steps."""
+    rng = np.random.default_rng(31_000 + case)
+    M = int(rng.choice([int(rng.integers(1, 65)), int(rng.choice([12, 20, 24, 28, 36, 40, 44, 48, 52, 56, 60, 64])),
+                        int(rng.choice([5, 6, 7, 9, 11, 13, 17, 31, 33, 63]))]))
+    P = int(rng.choice([int(rng.integers(1, 300)), int(rng.integers(300, 60_000))]))
+    variant = int(rng.integers(0, 3))
+    theta_kind = int(rng.integers(0, 3))
+    D = int(rng.integers(1, 4))
+    have = int(rng.integers(0, D + 1))
+    wire = [(0, 0, 0), (1, 0, 0), (2, 4, 3), (2, 5, 2), (2, 2, 1), (2, 3, 0), (2, 3, 2)][int(rng.integers(0, 7))]
+    eta, mu = float(rng.choice([0.4, 0.7, 1.0])), float(rng.choice([0.0, 0.5, 0.9]))
+    what = f"case {case}: M={M} P={P} variant={variant} kind={theta_kind} D={D} have={have} wire={wire}"
+    st = inputs.make_outer_state(M, P, 5000 + case, device=DEV, theta_kind=theta_kind, overlap_steps=D)
+    st["outer_mom"][:, :P].normal_(0.0, 1e-3, generator=st["gen"])
+    h = host_copy(st)
+    h["delta_prev_local"] = h["delta_prev_local"].reshape(D, M, st["stride"])
+    h["delta_prev_avg"] = h["delta_prev_avg"].reshape(D, st["stride"])
+    scratch = torch.zeros(64, dtype=torch.int32, device=DEV)
+    state = binding.State.from_dict(st, outer_lr=eta, outer_momentum=mu, have_prev=have, overlap_steps=D,
+                                    comm_scratch=scratch)
+    for k in range(D + 2):
+        if k:
+            inputs.inner_phase_standin(st)
+            h["theta"], h["master"] = to_numpy(st["theta"]), to_numpy(st["master"])
+        state.outer_quantized(variant, *wire)
+        have = oracle.outer_step_overlap(variant, k, have, M=M, P=P, stride=st["stride"], eta=eta, mu=mu,
+                                         theta=h["theta"], master=h["master"], start=h["start"],
+                                         outer_mom=h["outer_mom"], delta_prev_local=h["delta_prev_local"],
+                                         delta_prev_avg=h["delta_prev_avg"], theta_kind=theta_kind, comm=wire[0],
+                                         exp_bits=wire[1], man_bits=wire[2], nthreads=4)
+        torch.cuda.synchronize()
+        got = {key: st[key] for key in ("theta", "master", "start", "outer_mom")}
+        got["delta_prev_local"] = st["delta_prev_local"].view(D, M, st["stride"])
+        got["delta_prev_avg"] = st["delta_prev_avg"].view(D, st["stride"])
+        assert_state_equal(got, h, keys=tuple(got), what=f"{what} step {k + 1}")
+    state.close()
