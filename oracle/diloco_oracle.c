@@ -37,7 +37,9 @@
  *     2^(X-1)-1, subnormals, every code a finite number (no inf/NaN codes),
  *     round to nearest with ties to the even code, saturating; each replica's
  *     vector is scaled so that its largest magnitude maps to the format's
- *     largest value (one fp32 scale per replica per outer step).  PARITY
+ *     largest value (one fp32 scale per replica per outer step; the maximum
+ *     propagates NaN and a scale that is zero or underflows to zero is
+ *     replaced by 1, see amax_update / amax_to_scale).  PARITY
  *     UNPINNED against the paper for the EXMY layout and scaling (nothing is
  *     printed to pin them to); the rounding itself is pinned by brute force
  *     over every code, the E2M1 value table and a library's float8 casts.
@@ -144,7 +146,8 @@ static int exmy_code(double v, int X, int Y)
 static double exmy_round(double y, int X, int Y)
 {
     double a = fabs(y);
-    if (a == 0.0 || a != a) return y;
+    if (a == 0.0 || a != a) return y;  /* zero keeps its sign; NaN stays NaN */
+    if (isinf(a)) return y < 0 ? -exmy_max(X, Y) : exmy_max(X, Y); /* saturating, like any |y| > max */
     int bias = (1 << (X - 1)) - 1;
     int e2;
     (void)frexp(a, &e2);               /* a = f * 2^e2, 0.5 <= f < 1  =>  2^(e2-1) <= a */
@@ -160,6 +163,33 @@ static double exmy_round(double y, int X, int Y)
     double top = exmy_max(X, Y);
     if (q > top) q = top;
     return y < 0 ? -q : q;
+}
+
+/*
+ * Per-replica scale of the EXMY wire format.  amax = max_i |Delta_m[i]| where the maximum
+ * PROPAGATES NaN (as IEEE 754-2019 `maximum` does): one NaN element makes amax NaN.
+ * scale = amax / max(EXMY), except that a scale of zero (the replica did not move, or moved
+ * so little that the quotient underflows to zero in REAL) is replaced by 1.  Consequences,
+ * all by plain IEEE arithmetic in the lines below: a replica whose outer gradient holds a NaN
+ * or an infinity has a NaN or infinite scale, and EVERY element it puts on the wire decodes
+ * to NaN (x / NaN, 0 * inf): a non-finite outer gradient poisons that replica's whole
+ * contribution instead of being silently clamped to the format's largest value.  (A reading:
+ * the paper does not discuss non-finite values.  With the bf16 wire there is no scale and
+ * NaN / infinity travel element by element.)
+ */
+static REAL amax_update(REAL amax, REAL d)
+{
+    REAL ab = d < 0 ? -d : d;
+    if (ab != ab) return ab;            /* NaN enters ... */
+    if (amax != amax) return amax;      /* ... and stays */
+    return ab > amax ? ab : amax;
+}
+
+static REAL amax_to_scale(REAL amax, int X, int Y)
+{
+    REAL scale = amax / (REAL)exmy_max(X, Y);
+    if (scale == (REAL)0) scale = (REAL)1;
+    return scale;
 }
 
 /* what the wire carries for one element of replica m's outer gradient */
@@ -209,10 +239,9 @@ int FN(oracle_outer_step_comm)(int variant, int bootstrap, int M, int64_t P, int
             for (int64_t i = 0; i < P; ++i) {
                 size_t at = (size_t)m * (size_t)stride + (size_t)i;
                 REAL dm = start[at] - load_theta(theta_kind, theta, master, at);
-                REAL ab = dm < 0 ? -dm : dm;
-                if (ab > amax) amax = ab;
+                amax = amax_update(amax, dm);
             }
-            if (amax > (REAL)0) scale[m] = amax / (REAL)exmy_max(X, Y);
+            scale[m] = amax_to_scale(amax, X, Y);
             if (scales_out) scales_out[m] = scale[m];
         }
     }
@@ -304,17 +333,17 @@ int FN(oracle_wire_encode)(int64_t P, const REAL *d, int X, int Y, uint8_t *payl
 {
     if (P < 0 || X < 1 || X > 5 || Y < 0 || X + Y > 7) return -1;
     REAL amax = (REAL)0;
-    for (int64_t i = 0; i < P; ++i) {
-        REAL ab = d[i] < 0 ? -d[i] : d[i];
-        if (ab > amax) amax = ab;
-    }
-    REAL scale = amax > (REAL)0 ? amax / (REAL)exmy_max(X, Y) : (REAL)1;
+    for (int64_t i = 0; i < P; ++i) amax = amax_update(amax, d[i]);
+    REAL scale = amax_to_scale(amax, X, Y);
     const int packed = wire_packed(X, Y);
     if (packed) memset(payload, 0, (size_t)((P + 1) / 2));
     for (int64_t i = 0; i < P; ++i) {
         REAL y = d[i] / scale;
         double q = exmy_round((double)y, X, Y);
-        int code = exmy_code(fabs(q), X, Y) | ((signbit(q) ? 1 : 0) << (X + Y));
+        /* every code is a finite number, so NaN has none.  y is NaN only when this worker's
+           scale is NaN or infinite; it then travels as code 0 (+0), which the receiver's
+           value(code) * scale turns back into NaN (0 * NaN, 0 * inf): same result as the fused step */
+        int code = (q != q) ? 0 : exmy_code(fabs(q), X, Y) | ((signbit(q) ? 1 : 0) << (X + Y));
         if (packed) payload[i / 2] |= (uint8_t)(code << (4 * (i & 1)));
         else payload[i] = (uint8_t)code;
     }
@@ -344,7 +373,7 @@ int FN(oracle_wire_decode_sum)(int M, int64_t P, int64_t payload_stride, const u
         for (int m = 0; m < M; ++m) {
             const uint8_t *row = payloads + (size_t)m * (size_t)payload_stride;
             int code = packed ? (row[i / 2] >> (4 * (i & 1))) & 15 : row[i];
-            REAL scale = amaxes[m] > (REAL)0 ? amaxes[m] / (REAL)exmy_max(X, Y) : (REAL)1;
+            REAL scale = amax_to_scale(amaxes[m], X, Y);
             REAL w = (REAL)exmy_decode(code, X, Y) * scale;
             acc = (m == 0) ? w : acc + w;
         }

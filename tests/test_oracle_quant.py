@@ -263,3 +263,85 @@ def test_wire_round_trip_is_the_quantised_mean_of_the_step(oracle, X, Y):
     total = oracle.wire_decode_sum(np.stack(rows), np.array(amaxes, np.float32), P, X, Y)
     run(oracle, 2, st, comm=oracle.COMM_EXMY, exp_bits=X, man_bits=Y)
     np.testing.assert_array_equal(total / np.float32(M), st["delta_prev_avg"])
+
+
+# ---------------------------------------------------------------- non-finite and vanishing outer gradients
+@pytest.mark.parametrize("bad", [np.nan, np.inf, -np.inf])
+def test_non_finite_outer_gradient_poisons_the_replicas_scaled_contribution(oracle, bad):
+    """EXMY wire: max|Delta_m| propagates NaN and infinity, so the replica's scale is NaN or
+    infinite and every element it sends decodes to NaN (x / NaN, 0 * inf): the recorded mean
+    is NaN at EVERY index, not a clamped finite number.  The local, full-precision terms are
+    untouched: delta_prev_local holds the raw Delta_m.  bf16 wire (no scale): only the bad
+    index is non-finite."""
+    rng = np.random.default_rng(40)
+    M, P = 3, 64
+    st = state(rng, M, P)
+    st["theta"][1, 5] = bad                                    # Delta_1[5] = start - theta = -bad (or NaN)
+    d = st["start"] - st["theta"]
+    a = {k: v.copy() for k, v in st.items()}
+    scales = np.zeros(M, np.float32)
+    run(oracle, 2, a, comm=oracle.COMM_EXMY, exp_bits=4, man_bits=3, bootstrap=True, scales_out=scales)
+    assert np.isfinite(scales[0]) and np.isfinite(scales[2]) and not np.isfinite(scales[1])
+    assert np.isnan(scales[1]) == np.isnan(bad)
+    assert np.isnan(a["delta_prev_avg"]).all()
+    np.testing.assert_array_equal(a["delta_prev_local"], d)   # NaN == NaN positionally in this assert
+    b = {k: v.copy() for k, v in st.items()}
+    run(oracle, 2, b, comm=oracle.COMM_BF16, bootstrap=True)
+    finite = np.isfinite(b["delta_prev_avg"])
+    assert not finite[5] and finite.sum() == P - 1
+    # the rounding itself: NaN stays NaN, infinities saturate to the largest value
+    assert np.isnan(oracle.exmy_round(float("nan"), 4, 3))
+    assert oracle.exmy_round(float("inf"), 4, 3) == 480.0 and oracle.exmy_round(float("-inf"), 2, 1) == -6.0
+
+
+def test_scale_that_underflows_is_one_and_the_replica_sends_zeros(oracle):
+    """fp32 outer gradients so small that max|Delta_m| / max(EXMY) underflows to zero: the
+    scale is 1 (as for a replica that did not move), every element rounds to a zero of its own
+    sign, and the mean equals the mean of the other replicas' wire values divided by M."""
+    rng = np.random.default_rng(41)
+    M, P, X, Y = 2, 128, 4, 3
+    st = state(rng, M, P)
+    tiny = (rng.integers(-3, 4, P) * np.float32(1e-45)).astype(np.float32)   # multiples of the smallest subnormal
+    tiny[0] = np.float32(-0.0)
+    assert np.float32(np.abs(tiny).max()) / np.float32(480.0) == 0.0
+    st["start"][1] = 0.0
+    st["theta"][1] = -tiny                                     # Delta_1 = 0 - (-tiny) = tiny, exactly
+    ref = {k: v.copy() for k, v in st.items()}
+    ref["theta"][1] = ref["start"][1]                          # the same replica, not moved at all
+    scales = np.zeros(M, np.float32)
+    run(oracle, 1, st, comm=oracle.COMM_EXMY, exp_bits=X, man_bits=Y, bootstrap=True, scales_out=scales)
+    run(oracle, 1, ref, comm=oracle.COMM_EXMY, exp_bits=X, man_bits=Y, bootstrap=True)
+    assert scales[1] == 1.0
+    np.testing.assert_array_equal(st["delta_prev_avg"], ref["delta_prev_avg"])
+    # a subnormal scale that does not underflow is kept: amax = 2^-120, scale = 2^-120 / 480 > 0
+    st2 = state(rng, M, P)
+    st2["start"][1] = 0.0
+    st2["theta"][1] = 0.0
+    st2["theta"][1, 3] = -np.float32(2.0 ** -120)
+    run(oracle, 1, st2, comm=oracle.COMM_EXMY, exp_bits=X, man_bits=Y, bootstrap=True, scales_out=scales)
+    assert scales[1] == np.float32(2.0 ** -120) / np.float32(480.0) and 0 < scales[1] < 1.2e-38
+
+
+def test_wire_bytes_of_non_finite_outer_gradients(oracle):
+    """Every code is finite, so a NaN travels as code 0 next to a NaN (or infinite) maximum
+    word; decoding such a payload gives NaN everywhere (0 * NaN, 0 * inf), exactly what the
+    fused quantised step records."""
+    X, Y, P = 4, 3, 9
+    d = np.linspace(-1e-3, 1e-3, P).astype(np.float32)
+    d[4] = np.nan
+    payload, amax = oracle.wire_encode(d, X, Y)
+    assert np.isnan(amax) and (payload == 0).all()             # x / NaN is NaN for every element
+    d[4] = np.inf
+    payload, amax = oracle.wire_encode(d, X, Y)
+    assert np.isinf(amax) and payload[4] == 0                  # inf / inf
+    assert set(payload[np.arange(P) != 4]) <= {0x00, 0x80}     # finite / inf = a signed zero
+    other = np.full(P, 1e-3, np.float32)
+    p2, a2 = oracle.wire_encode(other, X, Y)
+    total = oracle.wire_decode_sum(np.stack([p2, payload]), np.array([a2, amax], np.float32), P, X, Y)
+    assert np.isnan(total).all()                               # 0 * inf
+    # ... which is the mean the fused quantised step records for the same two outer gradients
+    st = dict(start=np.zeros((2, P), np.float32), theta=-np.stack([other, d]),
+              delta_prev_local=np.zeros((2, P), np.float32), delta_prev_avg=np.zeros(P, np.float32),
+              outer_mom=np.zeros((2, P), np.float32))
+    run(oracle, 2, st, comm=oracle.COMM_EXMY, exp_bits=X, man_bits=Y, bootstrap=True)
+    assert np.isnan(st["delta_prev_avg"]).all()
