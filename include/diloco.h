@@ -32,7 +32,8 @@
  *     (a cudaStream_t cast to void*; NULL = the legacy default stream).  No call
  *     synchronises the device.  All buffers are updated in place.
  *   - every call returns a status (0 = DILOCO_OK, negative = error); nothing throws or
- *     aborts.  On error nothing has been launched and the state is unchanged.
+ *     aborts.  On error nothing has been launched and the state is unchanged (one exception,
+ *     stated there: a runtime failure in the middle of diloco_outer_step_host).
  *   - the device that was current at diloco_state_init must be current at every launching
  *     call on that state (DILOCO_ERR_BAD_STATE otherwise).
  *   - arithmetic: fp32, one IEEE round-to-nearest-even per operation, no FMA contraction,
@@ -221,10 +222,14 @@ int diloco_outer_quantized(diloco_state_t *state, int32_t variant, int32_t comm_
  * device.
  *
  * Limits and rules:
- *   - M <= DILOCO_MAX_M, else DILOCO_ERR_UNSUPPORTED (one word of scratch per replica).
+ *   - M <= DILOCO_MAX_M (64), else DILOCO_ERR_UNSUPPORTED: one word of scratch per replica
+ *     (diloco_state_init has the same limit today, so no existing state can exceed it).
+ *   - the device's ordinal must be below 64 (the library keeps one looked-up address per
+ *     ordinal), else DILOCO_ERR_UNSUPPORTED.
  *   - the state's device must be the current device, else DILOCO_ERR_BAD_STATE.
- *   - the first call on each device looks up the array's device address
+ *   - the first DILOCO_COMM_EXMY call on each device looks up the array's device address
  *     (cudaGetSymbolAddress) and keeps it; make that first call outside any stream capture.
+ *     The bf16 and fp32 formats reduce no maxima and never touch the array.
  *   - all states and all calls on a device share the one array.  The call clears the words
  *     it uses before reducing into them, so stale contents never matter, but two calls whose
  *     kernels can overlap on the GPU (different streams, no ordering between them) race on
@@ -324,6 +329,15 @@ int diloco_outer_fragment(diloco_state_t *state, int32_t variant, int32_t bootst
  * streams: three distinct cudaStream_t cast to void* (h2d, compute, d2h); chunk: elements
  * per chunk, a multiple of 64.  Returns after enqueueing; the caller synchronises streams[2].
  * Advances have_prev / outer-step counter like the device forms.
+ * Rows are moved one cudaMemcpyAsync per row and chunk, so rows of any length work.  Host
+ * memory that is not pinned is accepted but makes the copies synchronous with the host; a
+ * host_* pointer that is in fact device memory is refused (INVALID_ARG).
+ * Errors: arguments, buffers and everything else that can fail without touching a stream are
+ * checked before the first copy is enqueued, and such an error leaves the state unchanged.  If
+ * the CUDA runtime itself fails later, while chunks are being enqueued (DILOCO_ERR_CUDA from a
+ * copy, an event or a launch), earlier chunks are already in flight: the call returns at once,
+ * the counters are NOT advanced, and the state buffers on both sides are then a mixture of
+ * stepped and unstepped chunks - synchronise the three streams and restore from a checkpoint.
  */
 int diloco_outer_step_host(diloco_state_t *state, int32_t variant, const diloco_buffers_t *host,
                            void *const streams[3], int64_t chunk);
@@ -333,6 +347,24 @@ int diloco_state_get_counters(const diloco_state_t *state, int64_t *inner_step, 
 int diloco_state_set_counters(diloco_state_t *state, int64_t inner_step, int64_t outer_step, int32_t have_prev);
 int diloco_set_outer_hparams(diloco_state_t *state, float outer_lr, float outer_momentum);
 int diloco_set_impl(diloco_state_t *state, int32_t impl);
+
+/*
+ * Bound of the device-side waits.  Only DILOCO_IMPL_BULK waits on anything (an mbarrier that
+ * the TMA unit completes when a tile's rows have landed in shared memory); every such wait
+ * gives up after limit_ns nanoseconds of the GPU's global timer (0 selects the default, 1 s),
+ * the CTA then stops, gives its copies in flight one more limit to land, and the kernel
+ * reports through device_status (diloco_check_device_status -> DILOCO_ERR_DEVICE_TIMEOUT).  A
+ * kernel in which every wait runs out returns after about (ring depth 3 + 1) x limit_ns.
+ * After a time-out the step's results are invalid: the buffers hold a mixture of stepped and
+ * unstepped tiles, while have_prev and the outer-step counter have advanced as for a
+ * successful call; restore both from a checkpoint.
+ * test_extra_expect_bytes: 0 in production.  A multiple of 16, at most 1024: every tile's
+ * barrier is told to expect that many bytes more than the copies deliver, so every copy still
+ * lands but no wait ever completes.  It exists so that a test can drive the give-up path
+ * without faulting or hanging anything; with it set no tile is stepped and no state buffer is
+ * written.
+ */
+int diloco_set_wait_limit(diloco_state_t *state, uint64_t limit_ns, uint32_t test_extra_expect_bytes);
 
 /*
  * Read the state's device_status word (synchronises the given stream first).  Returns

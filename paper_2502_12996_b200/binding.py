@@ -71,6 +71,7 @@ SYMBOLS = {
     "diloco_state_set_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32]),
     "diloco_set_outer_hparams": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_float, ctypes.c_float]),
     "diloco_set_impl": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
+    "diloco_set_wait_limit": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32]),
     "diloco_check_device_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_launch_count": (ctypes.c_int64, []),
     "diloco_last_cuda_error": (ctypes.c_int32, []),
@@ -244,6 +245,9 @@ class State:
 
     def set_impl(self, impl) -> None:
         _check(load_library().diloco_set_impl(self._handle, impl), "diloco_set_impl")
+
+    def set_wait_limit(self, limit_ns, test_extra_expect_bytes=0) -> None:
+        _check(load_library().diloco_set_wait_limit(self._handle, limit_ns, test_extra_expect_bytes), "diloco_set_wait_limit")
 
     def check_device_status(self, stream=None) -> None:
         _check(load_library().diloco_check_device_status(self._handle, _stream_ptr(stream)), "diloco_check_device_status")

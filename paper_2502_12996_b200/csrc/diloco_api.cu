@@ -34,12 +34,15 @@ struct diloco_state {
   int64_t inner_step;
   int64_t outer_step;
   int32_t have_prev;
+  uint64_t wait_limit_ns;  // bound of every device-side wait of the bulk form
+  uint32_t test_extra_tx;  // bytes its barriers over-expect: 0 except in the give-up test
   std::vector<cudaEvent_t> events; // host-path chunk events, created on first use
   cudaEvent_t last_d2h;
 };
 
 // Scratch of diloco_outer_quantized_static: part of the library image, so every GPU that loads
 // the library holds these 64 words (256 bytes) until the process exits.
+constexpr uint64_t kDefaultWaitLimitNs = 1000000000ull; // 1 s per device-side wait
 constexpr int kStaticScratchWords = DILOCO_MAX_M;
 static __device__ __align__(256) unsigned g_static_scratch[kStaticScratchWords];
 
@@ -235,7 +238,7 @@ int launch_bulk_t(const diloco_state *st, const OuterArgs &a, cudaStream_t s) {
   long long grid = (long long)per_sm * st->sm_count;
   const long long ntiles = a.P / T;
   if (grid > ntiles) grid = ntiles;
-  k<<<(unsigned)grid, NT, smem, s>>>(a, st->buf.device_status);
+  k<<<(unsigned)grid, NT, smem, s>>>(a, st->buf.device_status, (unsigned long long)st->wait_limit_ns, st->test_extra_tx);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1);
@@ -440,6 +443,8 @@ int diloco_state_init(const diloco_config_t *config, const diloco_buffers_t *buf
   st->inner_step = 0;
   st->outer_step = 0;
   st->have_prev = config->have_prev;
+  st->wait_limit_ns = kDefaultWaitLimitNs;
+  st->test_extra_tx = 0;
   st->last_d2h = nullptr;
   *out = st;
   return DILOCO_OK;
@@ -532,11 +537,16 @@ int diloco_outer_quantized_static(diloco_state_t *st, int32_t variant, int32_t c
   if (comm_format == DILOCO_COMM_EXMY &&
       (exp_bits < 1 || exp_bits > 5 || man_bits < 0 || exp_bits + man_bits > 7))
     return DILOCO_ERR_INVALID_ARG;
-  if (st->cfg.M > kStaticScratchWords) return DILOCO_ERR_UNSUPPORTED; // one word of scratch per replica
-  unsigned *scratch = nullptr; // check_variant has verified that the state's GPU is the current one
-  rc = static_scratch_for_current_device(st->device, &scratch);
-  if (rc != DILOCO_OK) return rc;
+  // one word of scratch per replica; today no state can have more replicas than the array has
+  // words, the check keeps that true if the state limit is ever raised
+  if (st->cfg.M > kStaticScratchWords) return DILOCO_ERR_UNSUPPORTED;
   if (comm_format == DILOCO_COMM_F32) return outer_whole(st, variant, stream);
+  unsigned *scratch = nullptr; // only the EXMY formats reduce maxima; the others never touch the array
+  if (comm_format == DILOCO_COMM_EXMY) {
+    // check_variant has verified that the state's GPU is the current one
+    rc = static_scratch_for_current_device(st->device, &scratch);
+    if (rc != DILOCO_OK) return rc;
+  }
   // launch_outer_quantized zeroes the M words it reduces into before every use
   rc = launch_outer_quantized(st, variant, is_first_steps(st, variant), comm_format, exp_bits, man_bits, scratch,
                               static_cast<cudaStream_t>(stream));
@@ -700,9 +710,22 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
   for (const Leg &l : legs)
     if ((l.in || l.out) && !l.dev) return DILOCO_ERR_INVALID_ARG;
   if (!host->theta && !host->master) return DILOCO_ERR_INVALID_ARG; // something must come from the host
+  // a host buffer that is really device memory would turn the copies below into silent
+  // device-to-device copies of the wrong data: refuse it (unregistered host memory is accepted,
+  // the copies are then synchronous with respect to the host)
+  for (const Leg &l : legs) {
+    if (!l.hst || !(l.in || l.out)) continue;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, l.hst) != cudaSuccess) {
+      cudaGetLastError();
+      continue; // older drivers report plain malloc memory as an error: that is host memory
+    }
+    if (at.type == cudaMemoryTypeDevice) return DILOCO_ERR_INVALID_ARG;
+  }
   const int64_t P = st->cfg.P;
   const size_t nchunks = (size_t)((P + chunk - 1) / chunk);
   cudaError_t e;
+  // everything that can fail without touching a stream comes first
   while (st->events.size() < 2 * nchunks) {
     cudaEvent_t ev;
     e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
@@ -718,14 +741,25 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
     if (e != cudaSuccess) return cuda_fail(e);
   }
   const size_t row = (size_t)st->cfg.stride;
+  // One plain copy per row and chunk (rows of 2^29 fp32 elements and more exceed the pitch
+  // limit of the 2-D copy routines; chunks are megabytes, so the copies stay few and large).
+  auto copy_rows = [&](const Leg &l, int64_t off, int64_t len, bool to_device, cudaStream_t s) -> cudaError_t {
+    for (int r = 0; r < l.rows; ++r) {
+      const size_t at = ((size_t)r * row + (size_t)off) * l.elt;
+      char *dv = static_cast<char *>(l.dev) + at;
+      char *hs = static_cast<char *>(l.hst) + at;
+      cudaError_t ce = to_device ? cudaMemcpyAsync(dv, hs, (size_t)len * l.elt, cudaMemcpyHostToDevice, s)
+                                 : cudaMemcpyAsync(hs, dv, (size_t)len * l.elt, cudaMemcpyDeviceToHost, s);
+      if (ce != cudaSuccess) return ce;
+    }
+    return cudaSuccess;
+  };
   for (size_t c = 0; c < nchunks; ++c) {
     const int64_t off = (int64_t)c * chunk;
     const int64_t len = (off + chunk <= P) ? chunk : (P - off);
     for (const Leg &l : legs) {
       if (!l.in || !l.hst) continue; // a NULL host pointer: that buffer is resident on the device
-      e = cudaMemcpy2DAsync(static_cast<char *>(l.dev) + (size_t)off * l.elt, row * l.elt,
-                            static_cast<const char *>(l.hst) + (size_t)off * l.elt, row * l.elt,
-                            (size_t)len * l.elt, (size_t)l.rows, cudaMemcpyHostToDevice, s_in);
+      e = copy_rows(l, off, len, true, s_in);
       if (e != cudaSuccess) return cuda_fail(e);
     }
     e = cudaEventRecord(st->events[2 * c], s_in);
@@ -740,9 +774,7 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
     if (e != cudaSuccess) return cuda_fail(e);
     for (const Leg &l : legs) {
       if (!l.out || !l.hst) continue;
-      e = cudaMemcpy2DAsync(static_cast<char *>(l.hst) + (size_t)off * l.elt, row * l.elt,
-                            static_cast<const char *>(l.dev) + (size_t)off * l.elt, row * l.elt,
-                            (size_t)len * l.elt, (size_t)l.rows, cudaMemcpyDeviceToHost, s_out);
+      e = copy_rows(l, off, len, false, s_out);
       if (e != cudaSuccess) return cuda_fail(e);
     }
   }
@@ -779,6 +811,13 @@ int diloco_set_outer_hparams(diloco_state_t *st, float outer_lr, float outer_mom
 int diloco_set_impl(diloco_state_t *st, int32_t impl) {
   if (!st || impl < DILOCO_IMPL_AUTO || impl > DILOCO_IMPL_BULK) return DILOCO_ERR_INVALID_ARG;
   st->cfg.impl = impl;
+  return DILOCO_OK;
+}
+
+int diloco_set_wait_limit(diloco_state_t *st, uint64_t limit_ns, uint32_t test_extra_expect_bytes) {
+  if (!st || test_extra_expect_bytes % 16 != 0 || test_extra_expect_bytes > 1024) return DILOCO_ERR_INVALID_ARG;
+  st->wait_limit_ns = limit_ns ? limit_ns : kDefaultWaitLimitNs;
+  st->test_extra_tx = test_extra_expect_bytes;
   return DILOCO_OK;
 }
 

@@ -11,16 +11,25 @@
 //   all:       wait full[s] (bounded), update the tile in place, fence.proxy.async, barrier
 //   thread 0:  issue the row stores as one bulk group; before a stage is refilled, wait
 //              until the group that drained it has finished reading shared memory
-// Every wait is bounded: after kSpinLimit failed polls a thread raises the CTA's abort
-// flag, the CTA stops taking tiles, drains its own stores and reports through the
-// device status word (host: DILOCO_ERR_DEVICE_TIMEOUT).
+// Every wait is bounded in TIME: a thread that has polled a barrier for longer than the
+// launch's wait limit (nanoseconds of %globaltimer; 1 s unless the caller set another) raises
+// the CTA's abort flag, the CTA stops taking tiles, gives its loads in flight one more limit
+// to land, drains its own stores and reports through the device status word (host:
+// DILOCO_ERR_DEVICE_TIMEOUT).  Worst case a CTA therefore returns after (ring depth + 1) wait
+// limits.  A hard poll count backs the clock up.
 #pragma once
 #include "diloco_kernels.cuh"
 
 namespace diloco {
 
-constexpr unsigned kSpinLimit = 1u << 22; // polls of mbarrier.try_wait (each blocks up to a HW time slice)
+constexpr unsigned kSpinLimit = 1u << 26; // hard cap on polls of mbarrier.try_wait, whatever the clock says
 constexpr unsigned kStatusTimeout = 0x7101u;
+
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -76,8 +85,26 @@ template <int M, int VAR, int TK, int T> struct BulkStage {
   static constexpr unsigned kLoadBytes = (unsigned)offC; // everything before the bf16 copy is loaded
 };
 
+// Poll `bar` for the given phase until it completes, `limit_ns` has passed, the poll cap is hit
+// or (if `abort` is given) another thread of the CTA has given up.  Returns whether it completed.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, unsigned parity, unsigned long long limit_ns,
+                                                  const volatile unsigned *abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (unsigned spins = 0; spins < kSpinLimit; ++spins) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (abort && *abort) return false;
+    if (global_ns() - t0 > limit_ns) return false;
+  }
+  return false;
+}
+
+// limit_ns: how long one wait may last.  extra_tx: bytes added to what every tile's barrier
+// expects, 0 in production; a test sets it to make the waits run out (every copy still lands,
+// the barrier just never completes) and so exercise the give-up path without any fault.
 template <int M, int VAR, int TK, int T, int S, int NT>
-__global__ void __launch_bounds__(NT, 1) outer_step_bulk_kernel(const OuterArgs a, unsigned *status) {
+__global__ void __launch_bounds__(NT, 1) outer_step_bulk_kernel(const OuterArgs a, unsigned *status,
+                                                                unsigned long long limit_ns, unsigned extra_tx) {
   using L = BulkStage<M, VAR, TK, T>;
   static_assert(T % 8 == 0 && L::kBytes % 16 == 0, "rows must be multiples of 16 bytes");
   static_assert(S >= 3, "ring needs a current, a loading and a draining stage");
@@ -105,7 +132,7 @@ __global__ void __launch_bounds__(NT, 1) outer_step_bulk_kernel(const OuterArgs 
     unsigned char *st = smem + (size_t)(j % S) * L::kBytes;
     unsigned long long *bar = &full[j % S];
     const long long i0 = (blockIdx.x + j * gridDim.x) * T;
-    mbar_expect_tx(bar, L::kLoadBytes);
+    mbar_expect_tx(bar, L::kLoadBytes + extra_tx);
 #pragma unroll
     for (int m = 0; m < M; ++m) {
       const long long at = m * a.stride + i0;
@@ -150,13 +177,7 @@ __global__ void __launch_bounds__(NT, 1) outer_step_bulk_kernel(const OuterArgs 
     }
     // wait for this tile's rows, bounded
     {
-      unsigned long long *bar = &full[j % S];
-      const unsigned parity = (unsigned)((j / S) & 1);
-      unsigned spins = 0;
-      bool ok = false;
-      while (!(ok = mbar_try_wait(bar, parity))) {
-        if (++spins >= kSpinLimit || s_abort) break;
-      }
+      const bool ok = mbar_wait_bounded(&full[j % S], (unsigned)((j / S) & 1), limit_ns, &s_abort);
       if (!ok) s_abort = 1;
       else {
         unsigned char *st = smem + (size_t)(j % S) * L::kBytes;
@@ -234,10 +255,8 @@ __global__ void __launch_bounds__(NT, 1) outer_step_bulk_kernel(const OuterArgs 
     if (aborted) {
       if (tid == 0) {
         // give the loads still in flight a bounded chance to land before shared memory is released
-        for (long long q = j; q < mine && q <= j + LOOK; ++q) {
-          unsigned spins = 0;
-          while (!mbar_try_wait(&full[q % S], (unsigned)((q / S) & 1)) && ++spins < kSpinLimit) {}
-        }
+        for (long long q = j; q < mine && q <= j + LOOK; ++q)
+          mbar_wait_bounded(&full[q % S], (unsigned)((q / S) & 1), limit_ns, nullptr);
       }
       break;
     }

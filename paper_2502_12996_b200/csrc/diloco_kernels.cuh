@@ -210,24 +210,31 @@ __device__ __forceinline__ void nesterov(float g, float eta, float mu, float &b,
 // All scalings below are by powers of two and therefore exact in fp32.
 __device__ __forceinline__ float exmy_round(float y, const OuterArgs &a) {
   const float ay = fabsf(y);
-  if (ay == 0.f) return y;
-  int E = (int)((__float_as_uint(ay) >> 23) & 0xffu) - 127; // binade of |y| (fp32 subnormals: clamped next)
+  if (!(ay > 0.f)) return y;                                // zero keeps its sign, NaN stays NaN
+  const float ac = fminf(ay, a.fmt_max);                    // saturating: the largest value is a fixed point of
+                                                            // the rounding, and infinity never reaches the exponent
+  int E = (int)((__float_as_uint(ac) >> 23) & 0xffu) - 127; // binade of |y| (fp32 subnormals: clamped next)
   E = max(E, a.emin);                                       // below the smallest normal the spacing is fixed
   const int qe = E - a.man_bits;                            // spacing = 2^qe
-  const float n = ay * __uint_as_float((unsigned)(127 - qe) << 23); // |y| / spacing, exact
+  const float n = ac * __uint_as_float((unsigned)(127 - qe) << 23); // |y| / spacing, exact
   float r = rintf(n);                                       // halves go to the even integer = even code ...
   if (a.man_bits == 0 && n == 1.5f) r = ((E + a.bias) & 1) ? 2.f : 1.f; // ... except with no mantissa bits,
                                                             // where the code's parity is the exponent field's
-  float q = r * __uint_as_float((unsigned)(127 + qe) << 23);
-  q = fminf(q, a.fmt_max);
+  const float q = r * __uint_as_float((unsigned)(127 + qe) << 23);
   return copysignf(q, y);
 }
 
-// the per-replica scale: max |Delta_m| maps to the format's largest value (1 if the replica did not move)
+// The per-replica scale: max |Delta_m| maps to the format's largest value; a scale of zero
+// (the replica did not move, or so little that the quotient underflows) is replaced by 1.  The
+// maximum propagates NaN, so a replica whose outer gradient holds a NaN or an infinity gets a
+// NaN or infinite scale and everything it sends decodes to NaN (x / NaN, 0 * inf).
+__device__ __forceinline__ float amax_bits_to_scale(unsigned bits, float fmt_max) {
+  const float scale = __uint_as_float(bits) / fmt_max;
+  return scale == 0.f ? 1.f : scale;
+}
 __device__ __forceinline__ float comm_scale(const OuterArgs &a, int m) {
   if (a.comm != COMM_EXMY) return 1.f;
-  const float amax = __uint_as_float(a.amax[m]);
-  return amax > 0.f ? amax / a.fmt_max : 1.f;
+  return amax_bits_to_scale(a.amax[m], a.fmt_max);
 }
 
 // what replica m puts on the wire for one element of its outer gradient
@@ -238,12 +245,14 @@ __device__ __forceinline__ float comm_round(float d, float scale, const OuterArg
 }
 
 // Pass 1 of a quantised step: amax[m] = max_i |s_m[i] - theta_m[i]| (fp32, exact: max is
-// order-free).  grid = (blocks, M); non-negative floats order like their bit patterns.
+// order-free).  grid = (blocks, M).  The maximum is taken over the BIT PATTERNS of |Delta|:
+// non-negative floats order like their bit patterns, infinity sits above every finite value
+// and every NaN pattern above infinity, so one NaN element makes the result NaN.
 template <int TK, int NT, int U>
 __global__ void __launch_bounds__(NT) delta_amax_kernel(const OuterArgs a, unsigned *amax) {
   const int m = blockIdx.y;
   const long long nvec = a.P / 4;
-  float best = 0.f;
+  unsigned best = 0u;
   for (long long j0 = (long long)blockIdx.x * (NT * U) + threadIdx.x; j0 < nvec; j0 += (long long)gridDim.x * (NT * U)) {
     float s[U][4], x[U][4];
 #pragma unroll
@@ -260,24 +269,23 @@ __global__ void __launch_bounds__(NT) delta_amax_kernel(const OuterArgs a, unsig
 #pragma unroll
     for (int u = 0; u < U; ++u)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) best = fmaxf(best, fabsf(s[u][e] - x[u][e]));
+      for (int e = 0; e < 4; ++e) best = max(best, __float_as_uint(fabsf(s[u][e] - x[u][e])));
   }
   if (blockIdx.x == 0) {
     for (long long i = nvec * 4 + threadIdx.x; i < a.P; i += NT) {
       float s[1], x[1];
       F32Vec<1>::load(a.start + m * a.stride + i, s);
       load_theta<TK, 1>(a, m * a.stride + i, x);
-      best = fmaxf(best, fabsf(s[0] - x[0]));
+      best = max(best, __float_as_uint(fabsf(s[0] - x[0])));
     }
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
-  __shared__ float warp_best[NT / 32];
+  best = __reduce_max_sync(0xffffffffu, best);
+  __shared__ unsigned warp_best[NT / 32];
   if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
   __syncthreads();
   if (threadIdx.x == 0) {
-    for (int w = 1; w < NT / 32; ++w) best = fmaxf(best, warp_best[w]);
-    atomicMax(amax + m, __float_as_uint(best));
+    for (int w = 1; w < NT / 32; ++w) best = max(best, warp_best[w]);
+    atomicMax(amax + m, best);
   }
 }
 

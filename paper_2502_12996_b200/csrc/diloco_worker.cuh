@@ -133,16 +133,19 @@ struct WorkerQArgs {
 // EXMY code (without sign) and sign of y; same rounding as exmy_round
 __device__ __forceinline__ unsigned exmy_encode(float y, const WorkerQArgs &a) {
   const unsigned sign = (__float_as_uint(y) >> 31) << a.code_bits;
+  const unsigned top = (1u << a.code_bits) - 1u; // all exponent and mantissa bits set
   const float ay = fabsf(y);
   if (ay == 0.f) return sign;
-  int E = (int)((__float_as_uint(ay) >> 23) & 0xffu) - 127;
+  if (!(ay > 0.f)) return 0u;                    // NaN has no code; it arises only when this worker's scale is NaN
+                                                 // or infinite, and code 0 (+0) times that scale decodes to NaN
+  const float ac = fminf(ay, a.fmt_max);         // saturating
+  int E = (int)((__float_as_uint(ac) >> 23) & 0xffu) - 127;
   E = max(E, a.emin);
   const int qe = E - a.man_bits;
-  const float n = ay * __uint_as_float((unsigned)(127 - qe) << 23);
+  const float n = ac * __uint_as_float((unsigned)(127 - qe) << 23);
   float r = rintf(n);
   if (a.man_bits == 0 && n == 1.5f) r = ((E + a.bias) & 1) ? 2.f : 1.f;
   const float q = r * __uint_as_float((unsigned)(127 + qe) << 23);
-  const unsigned top = (1u << a.code_bits) - 1u; // all exponent and mantissa bits set
   if (q >= a.fmt_max) return sign | top;
   const unsigned ri = (unsigned)r;
   const unsigned one = 1u << a.man_bits;
@@ -162,8 +165,7 @@ __device__ __forceinline__ float exmy_decode(unsigned code, const WorkerQArgs &a
 }
 
 __device__ __forceinline__ float amax_to_scale(unsigned bits, float fmt_max) {
-  const float amax = __uint_as_float(bits);
-  return amax > 0.f ? amax / fmt_max : 1.f;
+  return amax_bits_to_scale(bits, fmt_max); // zero or underflowing scale -> 1; NaN and infinity propagate
 }
 
 // N consecutive elements starting at index i (N = 4 with i % 4 == 0, or N = 1): the codes of row m

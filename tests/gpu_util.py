@@ -66,14 +66,18 @@ def oracle_adamw(oracle, h, grads_np, M, P, stride, gstride, k, hp, theta_kind, 
 
 
 def bits(a):
-    """Bit patterns with +0 and -0 identified (IEEE equal; the sign of zero is not a result)."""
+    """Bit patterns with +0 and -0 identified (IEEE equal; the sign of zero is not a result) and
+    every NaN mapped to one pattern (which NaN an operation returns is not specified by IEEE
+    and differs between the host CPU and the GPU)."""
     if a.dtype == np.float32:
         u = a.view(np.uint32).copy()
         u[u == 0x80000000] = 0
+        u[(u & 0x7fffffff) > 0x7f800000] = 0x7fc00000
         return u
     if a.dtype == np.uint16:
         u = a.copy()
         u[u == 0x8000] = 0
+        u[(u & 0x7fff) > 0x7f80] = 0x7fc0
         return u
     return a
 

@@ -100,6 +100,46 @@ def test_bulk_staged_implementation(oracle, variant, theta_kind, M, P):
     run_outer_steps(oracle, variant, M, P, theta_kind, steps=3, seed=650 + M, impl=binding.IMPL_BULK)
 
 
+@pytest.mark.parametrize("M,P", [(2, 8 * 1024 + 5), (4, 40 * 512)])
+def test_bounded_device_wait_runs_out_and_is_reported(oracle, M, P):
+    """The staged form's only device-side waits are on mbarriers that the copy engine completes.
+    Here every barrier is told to expect 16 bytes more than its copies deliver: all copies land,
+    no wait can complete, every wait gives up after the 2 ms limit, the CTAs drain and return.
+    Nothing faults or hangs: the host reads the status word, gets DEVICE_TIMEOUT, finds the
+    state untouched, and the next ordinary call on a cleared status word equals the oracle."""
+    import time
+    st, checks = make(M, P, 660 + M, 0)
+    h = host_copy(st)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    state = binding.State.from_dict(st, impl=binding.IMPL_BULK, device_status=status)
+    state.set_wait_limit(2_000_000, 16)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    state.outer_eager()
+    with pytest.raises(binding.DilocoError) as e:
+        state.check_device_status()
+    elapsed = time.perf_counter() - t0
+    assert e.value.status == binding.ERR_DEVICE_TIMEOUT
+    assert int(status.item()) == 0x7101
+    assert 0.002 <= elapsed < 5.0, elapsed                     # at least one limit, at most a handful
+    assert_state_equal(st, h, what="after the timed-out launch")        # no tile was stepped
+    for bad in (8, 2048):
+        with pytest.raises(binding.DilocoError):
+            state.set_wait_limit(0, bad)
+    # recovery: same context, same state
+    status.zero_()
+    state.set_wait_limit(0, 0)
+    state.set_counters(0, 0, 1)
+    state.outer_eager()
+    oracle_outer(oracle, 2, h, M, P, st["stride"], 0.7, 0.9, 0)
+    state.check_device_status()
+    assert int(status.item()) == 0
+    assert_state_equal(st, h, what="ordinary call after the time-out")
+    for c in checks:
+        c()
+    state.close()
+
+
 @pytest.mark.parametrize("eta,mu", [(0.4, 0.9), (1.0, 0.0), (0.7, 0.0)])
 def test_other_outer_hyperparameters(oracle, eta, mu):
     run_outer_steps(oracle, 2, 4, 65_537, 0, steps=3, seed=700, eta=eta, mu=mu)
@@ -419,6 +459,42 @@ def test_host_entry_with_resident_optimizer_state(oracle):
     assert_state_equal(st, h, what="host path, device copy")
     with pytest.raises(binding.DilocoError):
         state.outer_step_host(binding.EAGER, binding.make_buffers(start=theta_host), streams, 64)
+    with pytest.raises(binding.DilocoError) as e:                # device memory where host memory belongs
+        state.outer_step_host(binding.EAGER, binding.make_buffers(theta=st["theta"].clone()), streams, 64 * 700)
+    assert e.value.status == binding.ERR_INVALID_ARG
+    assert state.get_counters()[1] == 1
+
+
+def test_host_entry_rows_longer_than_the_2d_copy_pitch_limit(oracle):
+    """Rows of 2^29 fp32 elements (2 GiB, the row length of the 550 M-parameter shapes and up)
+    exceed the pitch the 2-D copy routines accept; the host entry copies row by row.  Only P
+    elements per row are touched, so the buffers are allocated but never filled."""
+    M, P, stride = 2, 70_001, 1 << 29
+    if torch.cuda.mem_get_info()[0] < 24 << 30:
+        pytest.skip("needs 18 GiB of device memory")
+    small = inputs.make_outer_state(M, P, 1360, device=DEV)
+    st = dict(M=M, P=P, stride=stride, theta_kind=0, master=None, adam_m=None, adam_v=None)
+    for k in ("theta", "start", "delta_prev_local", "outer_mom"):
+        st[k] = torch.empty((M, stride), dtype=torch.float32, device=DEV)
+        st[k][:, :P] = small[k][:, :P]
+    st["delta_prev_avg"] = torch.empty(stride, dtype=torch.float32, device=DEV)
+    st["delta_prev_avg"][:P] = small["delta_prev_avg"][:P]
+    h = {k: (None if st.get(k) is None else st[k][..., :P].cpu().numpy().copy()) for k in
+         ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom")}
+    theta_host = torch.empty((M, stride), dtype=torch.float32)   # pageable, only P elements per row ever touched
+    theta_host[:, :P] = st["theta"][:, :P].cpu()
+    st["theta"][:, :P] = -7.0
+    state = binding.State.from_dict(st)
+    streams = [torch.cuda.Stream(device=DEV) for _ in range(3)]
+    state.outer_step_host(binding.EAGER, binding.make_buffers(theta=theta_host), streams, 64 * 300)
+    for s_ in streams:
+        s_.synchronize()
+    oracle.outer_step(oracle.EAGER, M=M, P=P, stride=P, eta=0.7, mu=0.9, theta=h["theta"], start=h["start"],
+                      outer_mom=h["outer_mom"], delta_prev_local=h["delta_prev_local"], delta_prev_avg=h["delta_prev_avg"])
+    got = {k: st[k][..., :P].contiguous() for k in ("start", "delta_prev_local", "delta_prev_avg", "outer_mom")}
+    got["theta"] = theta_host[:, :P].contiguous()
+    assert_state_equal(got, h, keys=tuple(got), what="host path, 2 GiB rows")
+    state.close()
 
 
 def test_launch_counter():
