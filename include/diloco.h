@@ -52,6 +52,7 @@ extern "C" {
 
 #define DILOCO_MAX_M 64
 #define DILOCO_MAX_OVERLAP 4
+#define DILOCO_MAX_FRAGMENTS 4096
 
 enum {
   DILOCO_OK = 0,
@@ -305,8 +306,8 @@ int diloco_worker_quantized_apply(diloco_state_t *state, int32_t variant, int32_
 
 /*
  * The same three steps restricted to parameter indices [offset, offset + len) of every
- * replica (a fragment, as Streaming DiLoCo applies the outer step to parts of the model
- * on different schedules, Section 3).  variant: 0 standard, 1 delayed, 2 eager.  bootstrap
+ * replica, with NO bookkeeping: the low-level form under diloco_outer_fragment_step (below),
+ * for callers that keep their own schedule state.  variant: 0 standard, 1 delayed, 2 eager.  bootstrap
  * != 0 performs the first-outer-step form for this fragment; the state's have_prev count is
  * NOT consulted and neither it nor the outer-step counter is changed: per-fragment
  * bookkeeping is the caller's (with overlap_steps > 1 the generation used is the one the
@@ -315,6 +316,34 @@ int diloco_worker_quantized_apply(diloco_state_t *state, int32_t variant, int32_
  */
 int diloco_outer_fragment(diloco_state_t *state, int32_t variant, int32_t bootstrap,
                           int64_t offset, int64_t len, void *cuda_stream);
+
+/*
+ * FRAGMENT SCHEDULES.  Streaming DiLoCo (Section 3, Experiments: the outer step is applied
+ * "to different parts of the models on different schedules"; appendix Table 4: fragments of
+ * three layers) gives every fragment of the parameter axis its own outer-step times.  Every
+ * index is independent of every other, so a fragment is just a range; what makes a schedule is
+ * that each fragment must remember on its own how many outer steps it has taken (which slot of
+ * the generation ring it reads and overwrites) and how many generations of its recorded
+ * gradients are valid (whether a delayed / eager step still only records, the t = H case).
+ *
+ * diloco_fragments_set: install a table of n fragments, fragment i = indices
+ *   [offsets[i], offsets[i] + lens[i]) of every replica; offsets multiples of 32 elements (64 if
+ *   theta is bf16), lens >= 1, inside [0, P), pairwise disjoint (they need not cover P).
+ *   offsets / lens are host arrays, copied.  Every fragment starts from the state's current
+ *   counters (outer-step counter and have_prev at the time of the call).  n = 0 removes the
+ *   table.  Errors: INVALID_ARG, MISALIGNED, UNSUPPORTED (n > DILOCO_MAX_FRAGMENTS).
+ * diloco_outer_fragment_step: one outer step (variant 0 standard, 1 delayed, 2 eager) of
+ *   fragment fragment_id, same kernel and arithmetic as the whole-vector calls.  Uses and
+ *   advances that fragment's counters only: while its have_prev < overlap_steps a delayed /
+ *   eager step records without applying, and with overlap_steps = D > 1 it consumes what this
+ *   fragment recorded D of ITS OWN outer steps ago.  The state's global counters are untouched.
+ * diloco_fragment_get_counters / _set_counters: per-fragment checkpoint / resume.
+ * Whole-vector calls and diloco_outer_fragment (below) ignore the table.
+ */
+int diloco_fragments_set(diloco_state_t *state, int32_t n, const int64_t *offsets, const int64_t *lens);
+int diloco_outer_fragment_step(diloco_state_t *state, int32_t variant, int32_t fragment_id, void *cuda_stream);
+int diloco_fragment_get_counters(const diloco_state_t *state, int32_t fragment_id, int64_t *outer_step, int32_t *have_prev);
+int diloco_fragment_set_counters(diloco_state_t *state, int32_t fragment_id, int64_t outer_step, int32_t have_prev);
 
 /*
  * End-to-end form of the three outer steps for callers whose state lives in HOST memory:
@@ -372,6 +401,45 @@ int diloco_set_wait_limit(diloco_state_t *state, uint64_t limit_ns, uint32_t tes
  * wait (its results are then invalid), DILOCO_ERR_CUDA on a runtime error.
  */
 int diloco_check_device_status(diloco_state_t *state, void *cuda_stream);
+
+/*
+ * COMPUTE-UTILISATION CALCULATOR (host only, no GPU work).  Section 3.1 and Table 2: a worker
+ * spends H * step_time_s computing per outer round and must move its outer gradient through its
+ * link once per round; with the all-reduce overlapped with the next D inner phases (D = 1:
+ * Algorithms 2-3, D = 2: "two-outer-steps" overlap) communication is free as long as it takes
+ * no longer than the TOLERATED LATENCY D * H * step_time_s (Table 2: 30 x 0.08 s = 2.4 s, and
+ * 4.8 s for D = 2; overlapping one inner step instead tolerates 0.08 s; blocking tolerates 0).
+ * Whatever exceeds it is idle time:
+ *     comm_time      = wire_bits / bandwidth_bit_s
+ *     exposed        = max(0, comm_time - tolerated_latency)
+ *     utilization    = compute_time / (compute_time + exposed)          (1 = never idle)
+ * wire_bits = P * bits_per_param, times 2 (M-1)/M if ring != 0 (what one worker sends in a ring
+ * all-reduce).  bits_per_param: 32, 16, or 8 * diloco_wire_payload_bytes(P, X, Y) / P for an EXMY
+ * wire.  This is the closed form the paper states in words; the figures of its Table 4 and
+ * Figure 4 come from a DAG simulator specified in another paper, which is NOT reproduced, so do
+ * not expect those numbers from this function.
+ * diloco_bandwidth_for_utilization inverts it: the smallest bandwidth (bit/s) that reaches the
+ * target utilisation in (0, 1] (bandwidth_bit_s of the input is ignored); INFINITY if none
+ * does (target 1 with nothing overlapped); a negative status cast to double on bad arguments.
+ * Errors: INVALID_ARG (null, P/M/H < 1, non-positive times, widths or bandwidth, negative
+ * overlaps, overlap_inner_steps > H or combined with overlap_outer_steps > 0).
+ */
+typedef struct {
+  int64_t P;                   /* parameters whose outer gradient is exchanged per outer step             */
+  double bits_per_param;       /* width of one outer-gradient element on the wire                         */
+  int32_t M;                   /* workers (matters only with ring != 0)                                   */
+  int32_t H;                   /* inner steps per outer step                                              */
+  double step_time_s;          /* pure compute time of one inner step                                     */
+  double bandwidth_bit_s;      /* link bandwidth per worker, bits per second (may be INFINITY)            */
+  int32_t overlap_outer_steps; /* D: 0 blocking (Algorithm 1), 1 Algorithms 2-3, 2 two-outer-steps, ...   */
+  int32_t overlap_inner_steps; /* with D = 0: inner steps the exchange is overlapped with (0 .. H)        */
+  int32_t ring;                /* 0: wire_bits = P * bits_per_param; 1: ring all-reduce factor 2 (M-1)/M  */
+} diloco_cu_input_t;
+typedef struct {
+  double wire_bits, comm_time_s, tolerated_latency_s, exposed_comm_time_s, compute_time_s, compute_utilization;
+} diloco_cu_output_t;
+int diloco_compute_utilization(const diloco_cu_input_t *in, diloco_cu_output_t *out);
+double diloco_bandwidth_for_utilization(const diloco_cu_input_t *in, double target_utilization);
 
 /* Number of kernels this library has launched in this process so far. */
 int64_t diloco_launch_count(void);

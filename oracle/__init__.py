@@ -123,6 +123,25 @@ def outer_step_overlap(variant, k, have, *, delta_prev_local=None, delta_prev_av
     return min(D, have + 1) if variant != STANDARD else have
 
 
+def outer_step_fragment(variant, k, have, offset, length, *, M, theta, start, outer_mom, delta_prev_local=None,
+                        delta_prev_avg=None, master=None, **kw):
+    """Outer step number ``k`` (0-based, counted per fragment) of the fragment made of indices
+    [offset, offset + length) of every replica, as Streaming DiLoCo steps parts of the model on
+    their own schedules (Section 3).  Every index is independent, so this is outer_step_overlap on
+    the slices: they are copied out, stepped, and copied back; nothing outside the fragment is
+    read or written.  ``delta_prev_local`` is [D, M, stride], ``delta_prev_avg`` [D, stride];
+    ``have`` counts the fragment's recorded generations.  Returns the fragment's new ``have``."""
+    sl = slice(offset, offset + length)
+    names = dict(theta=theta, start=start, outer_mom=outer_mom, delta_prev_local=delta_prev_local,
+                 delta_prev_avg=delta_prev_avg, master=master)
+    part = {n: (None if a is None else np.ascontiguousarray(a[..., sl])) for n, a in names.items()}
+    have = outer_step_overlap(variant, k, have, M=M, P=length, stride=length, **part, **kw)
+    for n, a in names.items():
+        if a is not None:
+            a[..., sl] = part[n]
+    return have
+
+
 def eager_gradient(form, *, M, P, stride, theta, start, delta_prev_local, delta_prev_avg=None,
                    master=None, theta_kind=THETA_NATIVE):
     """tilde-Delta_m for all m, without applying it: form 'a' = Alg. 3 line 11, 'b' = the

@@ -40,6 +40,19 @@ class Buffers(ctypes.Structure):
                 ("device_status", ctypes.c_void_p), ("comm_scratch", ctypes.c_void_p)]
 
 
+class CUInput(ctypes.Structure):
+    """diloco_cu_input_t"""
+    _fields_ = [("P", ctypes.c_int64), ("bits_per_param", ctypes.c_double), ("M", ctypes.c_int32), ("H", ctypes.c_int32),
+                ("step_time_s", ctypes.c_double), ("bandwidth_bit_s", ctypes.c_double),
+                ("overlap_outer_steps", ctypes.c_int32), ("overlap_inner_steps", ctypes.c_int32), ("ring", ctypes.c_int32)]
+
+
+class CUOutput(ctypes.Structure):
+    """diloco_cu_output_t"""
+    _fields_ = [(n, ctypes.c_double) for n in ("wire_bits", "comm_time_s", "tolerated_latency_s", "exposed_comm_time_s",
+                                               "compute_time_s", "compute_utilization")]
+
+
 class DilocoError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -66,6 +79,10 @@ SYMBOLS = {
     "diloco_worker_quantized_send": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_worker_quantized_apply": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "diloco_outer_fragment": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
+    "diloco_fragments_set": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)]),
+    "diloco_outer_fragment_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
+    "diloco_fragment_get_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)]),
+    "diloco_fragment_set_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int32]),
     "diloco_outer_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Buffers), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int64]),
     "diloco_state_get_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)]),
     "diloco_state_set_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32]),
@@ -73,6 +90,8 @@ SYMBOLS = {
     "diloco_set_impl": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32]),
     "diloco_set_wait_limit": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32]),
     "diloco_check_device_status": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_void_p]),
+    "diloco_compute_utilization": (ctypes.c_int, [ctypes.POINTER(CUInput), ctypes.POINTER(CUOutput)]),
+    "diloco_bandwidth_for_utilization": (ctypes.c_double, [ctypes.POINTER(CUInput), ctypes.c_double]),
     "diloco_launch_count": (ctypes.c_int64, []),
     "diloco_last_cuda_error": (ctypes.c_int32, []),
     "diloco_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -111,6 +130,30 @@ def wire_payload_bytes(P: int, exp_bits: int, man_bits: int) -> int:
     if n < 0:
         raise DilocoError(n, "diloco_wire_payload_bytes")
     return n
+
+
+def _cu_input(P, bits_per_param, M, H, step_time_s, bandwidth_bit_s, overlap_outer_steps, overlap_inner_steps, ring):
+    return CUInput(int(P), float(bits_per_param), int(M), int(H), float(step_time_s), float(bandwidth_bit_s),
+                   int(overlap_outer_steps), int(overlap_inner_steps), int(bool(ring)))
+
+
+def compute_utilization(*, P, bits_per_param, M, H, step_time_s, bandwidth_bit_s, overlap_outer_steps=1,
+                        overlap_inner_steps=0, ring=False) -> dict:
+    """diloco_compute_utilization: the output struct as a dict."""
+    inp = _cu_input(P, bits_per_param, M, H, step_time_s, bandwidth_bit_s, overlap_outer_steps, overlap_inner_steps, ring)
+    out = CUOutput()
+    _check(load_library().diloco_compute_utilization(ctypes.byref(inp), ctypes.byref(out)), "diloco_compute_utilization")
+    return {n: getattr(out, n) for n, _ in CUOutput._fields_}
+
+
+def bandwidth_for_utilization(target, *, P, bits_per_param, M, H, step_time_s, overlap_outer_steps=1,
+                              overlap_inner_steps=0, ring=False) -> float:
+    """diloco_bandwidth_for_utilization, bits per second."""
+    inp = _cu_input(P, bits_per_param, M, H, step_time_s, 1.0, overlap_outer_steps, overlap_inner_steps, ring)
+    w = float(load_library().diloco_bandwidth_for_utilization(ctypes.byref(inp), float(target)))
+    if w < 0:
+        raise DilocoError(int(w), "diloco_bandwidth_for_utilization")
+    return w
 
 
 def _check(status: int, where: str) -> None:
@@ -224,6 +267,25 @@ class State:
     def outer_fragment(self, variant, bootstrap, offset, length, stream=None) -> None:
         _check(load_library().diloco_outer_fragment(self._handle, variant, int(bool(bootstrap)), offset, length,
                                                     _stream_ptr(stream)), "diloco_outer_fragment")
+
+    def fragments_set(self, offsets, lens) -> None:
+        n = len(offsets)
+        a, b = (ctypes.c_int64 * max(n, 1))(*offsets), (ctypes.c_int64 * max(n, 1))(*lens)
+        _check(load_library().diloco_fragments_set(self._handle, n, a, b), "diloco_fragments_set")
+
+    def outer_fragment_step(self, variant, fragment_id, stream=None) -> None:
+        _check(load_library().diloco_outer_fragment_step(self._handle, variant, fragment_id, _stream_ptr(stream)),
+               "diloco_outer_fragment_step")
+
+    def fragment_get_counters(self, fragment_id):
+        a, b = ctypes.c_int64(), ctypes.c_int32()
+        _check(load_library().diloco_fragment_get_counters(self._handle, fragment_id, ctypes.byref(a), ctypes.byref(b)),
+               "diloco_fragment_get_counters")
+        return a.value, b.value
+
+    def fragment_set_counters(self, fragment_id, outer_step, have_prev) -> None:
+        _check(load_library().diloco_fragment_set_counters(self._handle, fragment_id, outer_step, int(have_prev)),
+               "diloco_fragment_set_counters")
 
     def outer_step_host(self, variant, host: Buffers, streams, chunk) -> None:
         arr = (ctypes.c_void_p * 3)(*[int(s.cuda_stream) for s in streams])

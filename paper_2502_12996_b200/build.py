@@ -46,7 +46,8 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
     from concurrent.futures import ThreadPoolExecutor
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     OBJ.mkdir(exist_ok=True)
-    jobs = [(CSRC / "diloco_api.cu", OBJ / "diloco_api.o", [])]
+    jobs = [(CSRC / "diloco_api.cu", OBJ / "diloco_api.o", []),
+            (CSRC / "diloco_utilization.cu", OBJ / "diloco_utilization.o", [])]
     jobs += [(CSRC / "diloco_outer_m.cu", OBJ / f"diloco_outer_m{m}.o", [f"DILOCO_M={m}"]) for m in OUTER_M]
     with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as pool:
         logs = list(pool.map(lambda j: _compile(nvcc, *j), jobs))

@@ -4,12 +4,14 @@
 // device synchronisation (except diloco_check_device_status), no CPU fallback.
 #include "../../include/diloco.h"
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "diloco_bulk.cuh"
@@ -26,6 +28,14 @@ using namespace diloco;
 DILOCO_FOR_EACH_M(DILOCO_EXTERN)
 #undef DILOCO_EXTERN
 
+// One fragment of the parameter axis with its own outer-step schedule (Streaming DiLoCo applies
+// the outer step to different parts of the model at different times, Section 3).
+struct Fragment {
+  int64_t offset, len;
+  int64_t outer_step; // outer steps this fragment has taken: selects its slot of the generation ring
+  int32_t have_prev;  // generations of its recorded gradients that are valid, 0 .. overlap_steps
+};
+
 struct diloco_state {
   diloco_config_t cfg;
   diloco_buffers_t buf;
@@ -34,6 +44,7 @@ struct diloco_state {
   int64_t inner_step;
   int64_t outer_step;
   int32_t have_prev;
+  std::vector<Fragment> frags;
   uint64_t wait_limit_ns;  // bound of every device-side wait of the bulk form
   uint32_t test_extra_tx;  // bytes its barriers over-expect: 0 except in the give-up test
   std::vector<cudaEvent_t> events; // host-path chunk events, created on first use
@@ -159,13 +170,13 @@ int check_variant(const diloco_state *st, int var) {
   return DILOCO_OK;
 }
 
-OuterArgs outer_args(const diloco_state *st, int64_t offset, int64_t len) {
+OuterArgs outer_args(const diloco_state *st, int64_t offset, int64_t len, int ring = -1) {
   OuterArgs a;
   const diloco_buffers_t &b = st->buf;
   a.theta = b.theta ? static_cast<char *>(b.theta) + (size_t)offset * theta_elt(st->cfg.theta_kind) : nullptr;
   a.master = b.master ? b.master + offset : nullptr;
   a.start = b.start + offset;
-  const size_t slot = (size_t)ring_slot(st);
+  const size_t slot = (size_t)(ring < 0 ? ring_slot(st) : ring);
   a.dpl = b.delta_prev_local ? b.delta_prev_local + slot * (size_t)st->cfg.M * (size_t)st->cfg.stride + offset : nullptr;
   a.dpa = b.delta_prev_avg ? b.delta_prev_avg + slot * (size_t)st->cfg.stride + offset : nullptr;
   a.mom = b.outer_mom + offset;
@@ -262,8 +273,8 @@ int launch_bulk_m(const diloco_state *st, int var, int tk, const OuterArgs &a, c
   return DILOCO_ERR_INVALID_ARG;
 }
 
-int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t len, cudaStream_t s) {
-  OuterArgs a = outer_args(st, offset, len);
+int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t len, cudaStream_t s, int ring = -1) {
+  OuterArgs a = outer_args(st, offset, len, ring);
   // The bulk form exists for M = 2 and M = 4 only, needs the status word for its bounded
   // waits and at least one full tile; everything else (and AUTO) takes the direct form,
   // which measured faster at every M.
@@ -674,6 +685,56 @@ int diloco_outer_fragment(diloco_state_t *st, int32_t variant, int32_t bootstrap
   const int64_t q = st->cfg.theta_kind == DILOCO_THETA_F32 ? 32 : 64;
   if (offset % q != 0) return DILOCO_ERR_MISALIGNED;
   return launch_outer(st, variant, bootstrap != 0, offset, len, static_cast<cudaStream_t>(stream));
+}
+
+int diloco_fragments_set(diloco_state_t *st, int32_t n, const int64_t *offsets, const int64_t *lens) {
+  if (!st || n < 0 || (n > 0 && (!offsets || !lens))) return DILOCO_ERR_INVALID_ARG;
+  if (n > DILOCO_MAX_FRAGMENTS) return DILOCO_ERR_UNSUPPORTED;
+  const int64_t q = st->cfg.theta_kind == DILOCO_THETA_F32 ? 32 : 64;
+  std::vector<Fragment> f((size_t)n);
+  for (int32_t i = 0; i < n; ++i) {
+    if (offsets[i] < 0 || lens[i] < 1 || offsets[i] > st->cfg.P - lens[i]) return DILOCO_ERR_INVALID_ARG;
+    if (offsets[i] % q != 0) return DILOCO_ERR_MISALIGNED;
+    f[(size_t)i] = Fragment{offsets[i], lens[i], st->outer_step, st->have_prev};
+  }
+  // fragments must not overlap: two schedules writing one index would make its history meaningless
+  std::vector<std::pair<int64_t, int64_t>> spans;
+  for (const Fragment &x : f) spans.emplace_back(x.offset, x.offset + x.len);
+  std::sort(spans.begin(), spans.end());
+  for (size_t i = 1; i < spans.size(); ++i)
+    if (spans[i].first < spans[i - 1].second) return DILOCO_ERR_INVALID_ARG;
+  st->frags.swap(f);
+  return DILOCO_OK;
+}
+
+int diloco_outer_fragment_step(diloco_state_t *st, int32_t variant, int32_t fragment_id, void *stream) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  int rc = check_variant(st, variant);
+  if (rc != DILOCO_OK) return rc;
+  if (fragment_id < 0 || (size_t)fragment_id >= st->frags.size()) return DILOCO_ERR_INVALID_ARG;
+  Fragment &f = st->frags[(size_t)fragment_id];
+  const bool boot = variant != VAR_STANDARD && f.have_prev < st->cfg.overlap_steps;
+  const int ring = (int)(f.outer_step % st->cfg.overlap_steps);
+  rc = launch_outer(st, variant, boot, f.offset, f.len, static_cast<cudaStream_t>(stream), ring);
+  if (rc != DILOCO_OK) return rc;
+  if (boot) f.have_prev += 1;
+  f.outer_step += 1;
+  return DILOCO_OK;
+}
+
+int diloco_fragment_get_counters(const diloco_state_t *st, int32_t fragment_id, int64_t *outer_step, int32_t *have_prev) {
+  if (!st || fragment_id < 0 || (size_t)fragment_id >= st->frags.size()) return DILOCO_ERR_INVALID_ARG;
+  if (outer_step) *outer_step = st->frags[(size_t)fragment_id].outer_step;
+  if (have_prev) *have_prev = st->frags[(size_t)fragment_id].have_prev;
+  return DILOCO_OK;
+}
+
+int diloco_fragment_set_counters(diloco_state_t *st, int32_t fragment_id, int64_t outer_step, int32_t have_prev) {
+  if (!st || fragment_id < 0 || (size_t)fragment_id >= st->frags.size()) return DILOCO_ERR_INVALID_ARG;
+  if (outer_step < 0 || have_prev < 0 || have_prev > st->cfg.overlap_steps) return DILOCO_ERR_INVALID_ARG;
+  st->frags[(size_t)fragment_id].outer_step = outer_step;
+  st->frags[(size_t)fragment_id].have_prev = have_prev;
+  return DILOCO_OK;
 }
 
 int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buffers_t *host, void *const streams[3],

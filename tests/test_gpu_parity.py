@@ -374,6 +374,93 @@ def test_fragments_equal_whole(oracle, theta_kind):
     assert e.value.status == binding.ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("D", [1, 2])
+@pytest.mark.parametrize("variant,theta_kind,impl", [(2, 0, 0), (2, 1, 0), (1, 2, 0), (0, 0, 0), (2, 0, 2)])
+def test_fragment_table_staggered_schedule(oracle, D, variant, theta_kind, impl):
+    """Streaming schedule: three fragments, fragment f takes its outer step at global steps
+    t = f mod 3, each with its own outer-step count (ring slot) and its own have_prev (its first
+    D eager / delayed steps only record).  The library keeps that state per fragment; the oracle
+    side runs the fragment helper with its own bookkeeping.  Bit-exact after every step."""
+    M, P = 4, 40_005
+    st = inputs.make_outer_state(M, P, 1150 + D, device=DEV, theta_kind=theta_kind, overlap_steps=D)
+    st["outer_mom"][:, :P].normal_(0.0, 1e-3, generator=st["gen"])
+    stride = st["stride"]
+    h = host_copy(st)
+    h["delta_prev_local"] = h["delta_prev_local"].reshape(D, M, stride)
+    h["delta_prev_avg"] = h["delta_prev_avg"].reshape(D, stride)
+    cuts = [(0, 64 * 200), (64 * 200, 64 * 300 + 1024), (64 * 500 + 1024, P - (64 * 500 + 1024))]
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    state = binding.State.from_dict(st, have_prev=0, overlap_steps=D, impl=impl, device_status=status)
+    state.fragments_set([c[0] for c in cuts], [c[1] for c in cuts])
+    have, count = [0, 0, 0], [0, 0, 0]
+    for t in range(3 * (D + 2)):
+        if t:
+            inputs.inner_phase_standin(st)
+            h["theta"], h["master"] = to_numpy(st["theta"]), to_numpy(st["master"])
+        f = t % 3
+        state.outer_fragment_step(variant, f)
+        have[f] = oracle.outer_step_fragment(variant, count[f], have[f], cuts[f][0], cuts[f][1], M=M, eta=0.7, mu=0.9,
+                                             theta=h["theta"], master=h["master"], start=h["start"],
+                                             outer_mom=h["outer_mom"], delta_prev_local=h["delta_prev_local"],
+                                             delta_prev_avg=h["delta_prev_avg"], theta_kind=theta_kind)
+        count[f] += 1
+        torch.cuda.synchronize()
+        got = {key: st[key] for key in ("theta", "master", "start", "outer_mom")}
+        got["delta_prev_local"] = st["delta_prev_local"].view(D, M, stride)
+        got["delta_prev_avg"] = st["delta_prev_avg"].view(D, stride)
+        assert_state_equal(got, h, keys=tuple(got), what=f"fragment schedule D={D} t={t} fragment {f}")
+        assert state.fragment_get_counters(f) == (count[f], have[f])
+    assert state.get_counters() == (0, 0, 0)                   # the whole-vector counters are not involved
+    state.check_device_status()
+    # resume: a fresh state with the fragments' counters restored continues identically
+    saved = [state.fragment_get_counters(f) for f in range(3)]
+    state.close()
+    state = binding.State.from_dict(st, have_prev=0, overlap_steps=D)
+    state.fragments_set([c[0] for c in cuts], [c[1] for c in cuts])
+    for f, (n, hv) in enumerate(saved):
+        state.fragment_set_counters(f, n, hv)
+    inputs.inner_phase_standin(st)
+    h["theta"], h["master"] = to_numpy(st["theta"]), to_numpy(st["master"])
+    state.outer_fragment_step(variant, 1)
+    oracle.outer_step_fragment(variant, count[1], have[1], cuts[1][0], cuts[1][1], M=M, eta=0.7, mu=0.9,
+                               theta=h["theta"], master=h["master"], start=h["start"], outer_mom=h["outer_mom"],
+                               delta_prev_local=h["delta_prev_local"], delta_prev_avg=h["delta_prev_avg"],
+                               theta_kind=theta_kind)
+    torch.cuda.synchronize()
+    got = {key: st[key] for key in ("theta", "master", "start", "outer_mom")}
+    got["delta_prev_local"] = st["delta_prev_local"].view(D, M, stride)
+    got["delta_prev_avg"] = st["delta_prev_avg"].view(D, stride)
+    assert_state_equal(got, h, keys=tuple(got), what="fragment schedule after resume")
+    state.close()
+
+
+def test_fragment_table_argument_checks():
+    st, _ = make(2, 10_000, 1160, 0, guards=False)
+    state = binding.State.from_dict(st)
+    for offs, lens, status in (([0, 64], [100, 10], binding.ERR_INVALID_ARG),       # overlap
+                               ([16], [10], binding.ERR_MISALIGNED),
+                               ([0], [0], binding.ERR_INVALID_ARG),
+                               ([9984], [100], binding.ERR_INVALID_ARG)):             # past P
+        with pytest.raises(binding.DilocoError) as e:
+            state.fragments_set(offs, lens)
+        assert e.value.status == status
+    with pytest.raises(binding.DilocoError) as e:
+        state.outer_fragment_step(binding.EAGER, 0)               # no table installed
+    assert e.value.status == binding.ERR_INVALID_ARG
+    state.fragments_set([0, 5024], [5000, 4976])
+    with pytest.raises(binding.DilocoError):
+        state.outer_fragment_step(binding.EAGER, 2)
+    with pytest.raises(binding.DilocoError):
+        state.fragment_set_counters(0, 0, 2)                       # have_prev > overlap_steps
+    state.outer_fragment_step(binding.EAGER, 1)
+    assert state.fragment_get_counters(1) == (1, 1) and state.fragment_get_counters(0) == (0, 1)
+    state.fragments_set([], [])
+    with pytest.raises(binding.DilocoError):
+        state.outer_fragment_step(binding.EAGER, 0)
+    torch.cuda.synchronize()
+    state.close()
+
+
 def test_resume_from_counters(oracle):
     """3 steps in one state == 1 step, state dropped, new state with restored counters, 2 steps."""
     M, P = 2, 50_001

@@ -113,3 +113,71 @@ def test_first_D_steps_only_record(oracle):
         np.testing.assert_array_equal(st["delta_prev_local"][k], d)
         assert not st["outer_mom"].any()
     assert have == D
+
+
+# ---------------------------------------------------------------- fragments on their own schedules
+def _frag_state(rng, D, M, P):
+    f = np.float32
+    s0 = rng.normal(0, 0.02, P)
+    st = dict(start=np.tile(s0, (M, 1)).astype(f), outer_mom=rng.normal(0, 1e-3, (M, P)).astype(f),
+              delta_prev_local=rng.normal(0, 1e-3, (D, M, P)).astype(f))
+    st["theta"] = (st["start"] + rng.normal(0, 1e-3, (M, P))).astype(f)
+    st["delta_prev_avg"] = st["delta_prev_local"].mean(1).astype(f)
+    return st
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("D", [1, 2])
+def test_fragments_stepped_together_equal_the_whole_vector(oracle, variant, D):
+    """All fragments of a partition stepped at the same outer step, in any order, give the bits
+    of one whole-vector step (slice independence, now through the fragment helper)."""
+    rng = np.random.default_rng(70 + D)
+    M, P = 3, 96
+    a = _frag_state(rng, D, M, P)
+    b = {k: v.copy() for k, v in a.items()}
+    cuts = [(64, 32), (0, 40), (40, 24)]
+    have_a, have_b = 0, [0, 0, 0]
+    for k in range(2 * D + 1):
+        if k:
+            noise = rng.normal(0, 1e-3, (M, P)).astype(np.float32)
+            a["theta"] = a["start"] + noise
+            b["theta"] = b["start"] + noise
+        have_a = oracle.outer_step_overlap(variant, k, have_a, M=M, P=P, stride=P, eta=0.7, mu=0.9, **a)
+        for f, (off, ln) in enumerate(cuts):
+            have_b[f] = oracle.outer_step_fragment(variant, k, have_b[f], off, ln, M=M, eta=0.7, mu=0.9, **b)
+        for key in a:
+            np.testing.assert_array_equal(a[key], b[key], err_msg=f"{key} step {k}")
+        assert have_b == [have_a] * 3
+
+
+def test_a_fragment_step_touches_only_its_fragment_and_schedules_commute(oracle):
+    """A step of one fragment leaves every index outside it untouched, bit for bit, so steps of
+    different fragments commute: a staggered schedule equals the same steps taken fragment by
+    fragment."""
+    rng = np.random.default_rng(75)
+    D, M, P = 2, 2, 128
+    st = _frag_state(rng, D, M, P)
+    thetas = [(st["start"] + rng.normal(0, 1e-3, (M, P))).astype(np.float32) for _ in range(6)]
+    cuts = [(0, 32), (32, 64), (96, 32)]
+    schedule = [(t, f) for t in range(6) for f in range(3) if t % 3 == f]            # staggered: fragment f at t = f mod 3
+
+    def run(order):
+        s = {k: v.copy() for k, v in st.items()}
+        have, count = [0, 0, 0], [0, 0, 0]
+        for t, f in order:
+            s["theta"] = thetas[t].copy()
+            off, ln = cuts[f]
+            before = {k: v.copy() for k, v in s.items()}
+            have[f] = oracle.outer_step_fragment(2, count[f], have[f], off, ln, M=M, eta=0.7, mu=0.9, **s)
+            count[f] += 1
+            outside = np.ones(P, bool)
+            outside[off:off + ln] = False
+            for key in s:
+                np.testing.assert_array_equal(s[key][..., outside], before[key][..., outside])
+        return s
+
+    a = run(schedule)
+    # theta is an input of each step (set from the same list), so compare what the steps own
+    b = run(sorted(schedule, key=lambda tf: (tf[1], tf[0])))
+    for key in ("start", "outer_mom", "delta_prev_local", "delta_prev_avg"):
+        np.testing.assert_array_equal(a[key], b[key], err_msg=key)
