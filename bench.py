@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the DiLoCo outer step with eager updates (and the kernels around it) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4a] [--impl ours|reference]
 
 One "step" is one fused eager outer step (Algorithm 3, lines 7-12: local outer gradients,
 M-way mean, eager combination, Nesterov update, replica reset) over all M replicas of the
@@ -9,11 +9,15 @@ workload; between steps an untimed stand-in for the inner phase moves the replic
 (theta_m <- start_m + N(0, 1e-3)) and a 256 MB buffer is written to flush L2.  For the
 phase workloads (cfg2, cfg3) a step is H fused AdamW steps followed by the eager outer step.
 
-Prints ONE JSON line.  `value` is flat parameters advanced per second (P / t), whole job
-(sum over ranks); `roofline` compares the algorithmic bytes of the dominant kernel with the
-measured HBM copy peak; `e2e` is the same step through diloco_outer_step_host with the state
-in pinned host memory (copies inside the timed region); `cpu_baseline` is the CPU oracle
-timed on this machine's host cores.
+The default workload is the largest outer-step shape of the five configurations that fits one
+GPU (cfg4a: M = 2, P = 2.4e9 fp32, 86 GB of state).  Prints ONE JSON line.  `value` is flat
+parameters advanced per second (P / t), whole job (sum over ranks); `roofline` compares the
+algorithmic bytes of the dominant kernel with the measured HBM copy peak; `e2e` is the same
+step through diloco_outer_step_host with the state in pinned host memory (copies inside the
+timed region); `cpu_baseline` is the CPU oracle timed on this machine's host cores; `shapes`
+(default single-GPU run only) holds the same kernel measurements for every other headline
+shape - cfg1, cfg4b, cfg4c, the cfg2 and cfg3 phases, cfg0 cold and warm - each with the
+clock samples of its own timed region.
 
 With --impl reference the CPU oracle itself is timed on the same workload (there is no
 reference implementation of this path; the paper ships no code).
@@ -21,6 +25,7 @@ reference implementation of this path; the paper ships no code).
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
 import subprocess
@@ -36,14 +41,12 @@ METRIC = "outer_step_params_per_s"
 UNIT = "params/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per parameter index for one launch of the
-# dominant kernel, from the captures summarised under profiles/ (None: not captured yet).
-NCU_TRAFFIC_BYTES_PER_PARAM = {
-    ("diloco_outer_eager", 4, 0): 134.38,    # profiles/outer_eager_f32_M4_P35M_cfg1.md
-    ("diloco_inner_adamw", 4, 1): 86.35,     # profiles/inner_adamw_bf16_M4_P35M_cfg2slice.md (35 M slice, scaled by P)
-    ("diloco_outer_eager", 16, 0): 516.2,    # profiles/outer_eager_f32_M16_P15M.md (15 M slice, scaled by P)
-}
+L2_BYTES = 126 << 20
+DEFAULT_WORKLOAD = "cfg4a"
+THETA_NAMES = ["f32", "bf16", "f32 master + bf16 copy"]
+VARIANTS = {"standard": 0, "delayed": 1, "eager": 2}
+# measured DRAM traffic per parameter index, one row per profiled kernel form
+TRAFFIC_TABLE = ROOT / "profiles" / "ncu_dram_bytes_per_index.txt"
 
 
 def outer_bytes_per_param(variant: int, M: int, theta_kind: int) -> int:
@@ -64,6 +67,11 @@ def adamw_bytes_per_param(M: int, theta_kind: int, grad_kind: int) -> int:
     return M * (th + g + 16)                          # + moments read+write
 
 
+def state_bytes_per_param(M: int, theta_kind: int, variant: int = 2) -> int:
+    th = {0: 4, 1: 2, 2: 6}[theta_kind]
+    return M * (th + 8 + (4 if variant == 2 else 0)) + (4 if variant else 0)
+
+
 def load_peak():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -74,8 +82,24 @@ def load_peak():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+def load_traffic():
+    """(kernel, variant, M, theta_kind) -> (DRAM bytes per index from an ncu capture, source).
+    The table is plain text: kernel variant M theta_kind bytes_per_index source."""
+    table = {}
+    try:
+        for line in TRAFFIC_TABLE.read_text().splitlines():
+            f = line.split()
+            if len(f) < 6 or line.lstrip().startswith("#"):
+                continue
+            table[(f[0], f[1], int(f[2]), int(f[3]))] = (float(f[4]), f[5])
+    except OSError:
+        pass
+    return table
+
+
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled every 100 ms from the warm-up on; the timed region's own samples are used when there are at least three."""
+    """nvidia-smi clocks and throttle reasons sampled every 100 ms for the whole run; every timed
+    region asks for the samples of its own window."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -95,15 +119,12 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
 
-    def stop(self, t0: float, t1: float, t_fallback: float = None):
+    def window(self, t0: float, t1: float, t_fallback: float = None):
+        """Median SM clock and the throttle reasons seen between t0 and t1 (a region shorter than
+        three samples falls back to the window that began with its warm-up, at t_fallback)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.25)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
         rows = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.25]
         window = "timed region"
         if len(rows) < 3 and t_fallback is not None:       # under load since the warm-up began
@@ -111,12 +132,13 @@ class ClockSampler:
             window = "warm-up + timed region"
         if not rows:
             rows, window = [r for (_, r) in self.rows], "whole run"
-        mhz, mx, reasons = [], None, set()
+        mhz, mx, watts, reasons = [], None, [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             try:
                 mhz.append(float(r[0]))
                 mx = float(r[1])
+                watts.append(float(r[2]))
             except Exception:
                 continue
             for n, v in zip(names, r[4:8]):
@@ -124,7 +146,16 @@ class ClockSampler:
                     reasons.add(n)
         mhz.sort()
         return {"sm_mhz": (mhz[len(mhz) // 2] if mhz else None), "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(mhz), "window": window}
+                "power_w_max": (max(watts) if watts else None), "samples": len(mhz), "window": window}
+
+    def stop(self):
+        if self.proc is None:
+            return
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
 
 
 def cpu_model() -> str:
@@ -135,6 +166,16 @@ def cpu_model() -> str:
     except OSError:
         pass
     return "unknown"
+
+
+def mem_available_bytes() -> int:
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 0
 
 
 def dist_env():
@@ -148,6 +189,21 @@ def shard_bounds(P_total: int, world: int, rank: int, quantum: int = 64):
     lo = (q * rank // world) * quantum
     hi = min(P_total, (q * (rank + 1) // world) * quantum)
     return lo, hi
+
+
+def config_dict(args, w, P_per_gpu: int) -> dict:
+    """What the workload is; the same dict in both arms (GPU path and CPU reference)."""
+    phase = w.H > 0 and not args.outer_only
+    state = state_bytes_per_param(w.M, w.theta_kind) * P_per_gpu
+    l2 = ("state >> 126 MB L2" if state > 4 * L2_BYTES else "state fits the 126 MB L2: cold-L2 figure") \
+        + ", 256 MB flush write before every timed step"
+    return {"workload": args.workload, "variant": args.variant, "M": w.M, "P_per_gpu": P_per_gpu,
+            "theta": THETA_NAMES[w.theta_kind],
+            "step": (f"{w.H} x inner AdamW + 1 outer {args.variant}" if phase else f"1 outer {args.variant} step"),
+            "outer_lr": w.outer_lr, "outer_momentum": w.outer_momentum, "l2": l2,
+            "sharding": "one full shape per rank (weak scaling), all M replicas of an index on one rank, no collective"
+            if not args.strong else "parameter axis split across ranks, all M replicas of an index on one rank, no collective",
+            "kernel_impl": ["auto", "direct", "bulk"][args.kernel], "outer_gradient_wire_format": args.comm}
 
 
 # ------------------------------------------------------------------------------------ CPU arm
@@ -186,6 +242,13 @@ def host_state(w, P, seed):
     return st, h
 
 
+def oracle_sample_size(w, P: int) -> int:
+    """Bounded sample of a workload for the CPU oracle: the per-parameter cost of the elementwise
+    path does not depend on P, so large shapes are timed on the first 1.4e8 / M parameters of
+    every replica (a few seconds per step on 16 cores)."""
+    return min(P, 140_000_000 // w.M)
+
+
 def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
@@ -194,30 +257,267 @@ def run_reference(args):
     from paper_2502_12996_b200 import inputs
     oracle.build()
     w = inputs.WORKLOADS[args.workload]
-    P = args.P or min(w.P, 35_000_000)                     # bounded sample of larger workloads
+    P_cfg = args.P or w.P
+    P = oracle_sample_size(w, P_cfg)
     cores = os.cpu_count() or 1
     st, h = host_state(w, P, w.seed)
     stride = st["stride"]
-    for _ in range(max(1, args.warmup)):
+    for _ in range(max(1, min(args.warmup, 3))):
         time_oracle_eager(h, w.M, P, stride, w.theta_kind, w.outer_lr, w.outer_momentum, cores, 0, 1)
     times = time_oracle_eager(h, w.M, P, stride, w.theta_kind, w.outer_lr, w.outer_momentum, cores, 1e9, args.steps)
     ms = 1e3 * sum(times) / len(times)
     value = P / (ms * 1e-3)
-    sample = f"eager outer step, M={w.M}, P={P} of {w.P} (all replicas), {len(times)} steps, {cores} OpenMP threads"
+    sample = (f"eager outer step on the first {P} of {P_cfg} parameters of all {w.M} replicas "
+              f"({len(times)} steps, {cores} OpenMP threads); per-parameter cost does not depend on P")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "variant": "eager", "M": w.M, "P": P, "theta": ["f32", "bf16", "f32 master + bf16 copy"][w.theta_kind]},
+            "dtype": "f32", "data": "synthetic", "config": config_dict(args, w, P_cfg),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
                              "cpu_model": cpu_model()},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0,
-            "note": "the paper ships no code: the reference arm is the CPU oracle (plain C, -O2, no FMA) on the host cores"}
+            "note": "the paper ships no code: the reference arm is the CPU oracle (plain C, -O2, no FMA) on the host cores; "
+                    "ms_per_step is the time of one step over the sample"}
     print(json.dumps(line))
     return 0
 
 
 # ------------------------------------------------------------------------------------ GPU arm
+COMM = {"f32": (0, 0, 0), "bf16": (1, 0, 0), "e4m3": (2, 4, 3), "e5m2": (2, 5, 2), "e2m1": (2, 2, 1), "e3m0": (2, 3, 0)}
+
+
+def stats(xs):
+    s = sorted(xs)
+    return {"mean": sum(s) / len(s), "median": s[len(s) // 2], "min": s[0], "max": s[-1], "n": len(s)}
+
+
+class Shape:
+    """One workload resident on the device: state, library handle, gradients, and the timed loop."""
+
+    def __init__(self, name, args, dev, rank, world, P=None, phase=None, variant=None, comm="f32"):
+        import torch
+        from paper_2502_12996_b200 import binding, inputs
+        self.torch, self.binding, self.inputs = torch, binding, inputs
+        self.name, self.dev = name, dev
+        w = self.w = inputs.WORKLOADS[name]
+        self.P = P or w.P
+        if args.strong and P is None:
+            lo, hi = shard_bounds(self.P, world, rank)
+            self.P = hi - lo
+        self.variant = VARIANTS[args.variant] if variant is None else variant
+        self.phase = (w.H > 0 and not args.outer_only) if phase is None else phase
+        self.comm = COMM[comm]
+        self.kernel = args.kernel
+        self.seed = w.seed + 1000 * rank
+        self.st = self.state = self.grads = self.scratch = None
+
+    def need_bytes(self):
+        w, M, P = self.w, self.w.M, self.P
+        th = {0: 4, 1: 2, 2: 6}[w.theta_kind]
+        per = th + 12 + ((8 + (2 if w.grad_kind else 4)) if self.phase else 0)
+        # state + one [M, P] fp32 temporary of the generator + stand-in chunks + the L2 flush buffer
+        return M * P * per + 4 * P + M * P * 4 + (768 << 20)
+
+    def fits(self):
+        free = self.torch.cuda.mem_get_info(self.dev)[0]
+        need = self.need_bytes()
+        return (need <= free), f"needs {need / 2**30:.1f} GiB of device memory, {free / 2**30:.1f} GiB free"
+
+    def allocate(self):
+        torch, binding, inputs, w = self.torch, self.binding, self.inputs, self.w
+        st = self.st = inputs.make_outer_state(w.M, self.P, self.seed, device=self.dev, theta_kind=w.theta_kind,
+                                               with_adam=self.phase)
+        kw = dict(H=w.H, outer_lr=w.outer_lr, outer_momentum=w.outer_momentum, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                  weight_decay=w.weight_decay, grad_kind=w.grad_kind, impl=self.kernel)
+        if self.comm[0]:
+            self.scratch = torch.zeros(64, dtype=torch.int32, device=self.dev)
+            kw["comm_scratch"] = self.scratch
+        self.state = binding.State.from_dict(st, **kw)
+        if self.phase:
+            if w.segments:
+                self.grads = torch.zeros((w.M, st["stride"]), dtype=torch.bfloat16 if w.grad_kind else torch.float32,
+                                         device=self.dev)
+                inputs.make_segment_grads(w.M, inputs.segment_sizes(self.P, w.segments),
+                                          inputs.segment_scales(w.segments, st["gen"], self.dev).tolist(), st["gen"],
+                                          self.grads)
+            else:
+                self.grads = inputs.make_grads(w.M, self.P, st["stride"], st["gen"], self.dev, w.grad_kind)
+        return self
+
+    def free(self):
+        if self.state is not None:
+            self.state.close()
+        self.st = self.state = self.grads = self.scratch = None
+        gc.collect()
+        self.torch.cuda.empty_cache()
+
+    def run_outer(self):
+        if self.comm[0]:
+            self.state.outer_quantized(self.variant, *self.comm)
+        else:
+            self.state.outer(self.variant)
+
+    def one_step(self, flush, timed=True, move=True, do_flush=True):
+        """(ms of the whole step, ms of the outer kernel, ms of the H AdamW steps), CUDA events on
+        the launching stream; the stand-in for the inner phase and the L2 flush are outside them."""
+        torch = self.torch
+        if not self.phase and move:
+            self.inputs.inner_phase_standin(self.st)
+        if do_flush:
+            flush.fill_(1)
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record()
+        if self.phase:
+            for _ in range(self.w.H):
+                self.state.inner_adamw(self.grads, self.w.inner_lr)
+        e1.record()
+        self.run_outer()
+        e2.record()
+        if not timed:
+            return None
+        e2.synchronize()
+        return e0.elapsed_time(e2), e1.elapsed_time(e2), e0.elapsed_time(e1)
+
+    def bytes_per_param(self):
+        w = self.w
+        outer = outer_bytes_per_param(self.variant, w.M, w.theta_kind)
+        if self.comm[0] == 2:                                    # the max-|Delta_m| pass re-reads theta and start
+            outer += w.M * ({0: 4, 1: 2, 2: 4}[w.theta_kind] + 4)
+        return outer, adamw_bytes_per_param(w.M, w.theta_kind, w.grad_kind)
+
+    def measure(self, flush, sampler, steps, warmup, barrier=None, move=True, do_flush=True):
+        """warmup untimed steps, then `steps` timed ones; returns the per-step rows, the launch
+        count of the timed region and the clock samples of that region."""
+        torch, binding = self.torch, self.binding
+        t_warm = time.perf_counter()
+        for _ in range(warmup):
+            self.one_step(flush, timed=False, move=move, do_flush=do_flush)
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        n0 = binding.launch_count()
+        t0 = time.perf_counter()
+        rows = [self.one_step(flush, move=move, do_flush=do_flush) for _ in range(steps)]
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        launches = binding.launch_count() - n0
+        if barrier:
+            barrier()
+        return rows, launches, sampler.window(t0, t1, t_warm)
+
+    def record(self, rows, clocks, peak, traffic):
+        """The figures of one shape as they go into the JSON line."""
+        w, P = self.w, self.P
+        outer_bpp, adam_bpp = self.bytes_per_param()
+        outer = stats([r[1] for r in rows])
+        vname = [k for k, v in VARIANTS.items() if v == self.variant][0]
+
+        def kernel(name, ms, bpp, key):
+            gbs = bpp * P / (ms["mean"] * 1e-3) / 1e9
+            tr = traffic.get(key)
+            return {"kernel": name, "ms": ms, "algorithmic_bytes_per_param": bpp, "GBps": gbs, "frac": gbs / peak,
+                    "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS, "GBps_best": bpp * P / (ms["min"] * 1e-3) / 1e9,
+                    "ncu_dram_bytes_per_param": (tr[0] if tr else None), "ncu_profile": (tr[1] if tr else None)}
+        rec = {"M": w.M, "P": P, "theta": THETA_NAMES[w.theta_kind], "state_GB": state_bytes_per_param(w.M, w.theta_kind) * P / 1e9,
+               "step_ms": stats([r[0] for r in rows]), "params_per_s": P / (sum(r[0] for r in rows) / len(rows) * 1e-3),
+               "outer": kernel(f"diloco_outer_{vname}", outer, outer_bpp,
+                               ("outer", vname, w.M, w.theta_kind) if not self.comm[0] else None),
+               "clocks": clocks}
+        if self.phase:
+            adam = stats([r[2] / w.H for r in rows])
+            rec["adamw"] = kernel("diloco_inner_adamw", adam, adam_bpp, ("adamw", "-", w.M, w.theta_kind))
+            rec["step"] = f"{w.H} x inner AdamW + 1 outer {vname}"
+        else:
+            rec["step"] = f"1 outer {vname} step"
+        return rec
+
+
+def register_host(torch, t):
+    """Page-lock a host tensor in place (exact size: the caching pinned allocator rounds every
+    request up to a power of two, which would double an 86 GB state)."""
+    rc = torch.cuda.cudart().cudaHostRegister(t.data_ptr(), t.numel() * t.element_size(), 0)
+    if int(rc) != 0:
+        raise RuntimeError(f"cudaHostRegister failed with {rc}")
+
+
+def unregister_host(torch, t):
+    torch.cuda.cudart().cudaHostUnregister(t.data_ptr())
+
+
+def run_e2e(shape, args, world, dist, red_dev, n_steps):
+    """The same outer step through diloco_outer_step_host: the state lives in pinned HOST memory,
+    every step copies what the step reads to the device, runs the kernel chunk by chunk and
+    copies what it wrote back, all inside the timed region."""
+    torch, binding = shape.torch, shape.binding
+    st, w, P, M, variant = shape.st, shape.w, shape.P, shape.w.M, shape.variant
+    keys = ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom")
+    pinned, t_pin = {}, time.perf_counter()
+    try:
+        for k in keys:
+            if st.get(k) is None:
+                pinned[k] = None
+                continue
+            pinned[k] = torch.empty(st[k].shape, dtype=st[k].dtype, device="cpu")
+            register_host(torch, pinned[k])
+            pinned[k].copy_(st[k])
+        t_pin = time.perf_counter() - t_pin
+        host = binding.make_buffers(**pinned)
+        streams = [torch.cuda.Stream(device=shape.dev) for _ in range(3)]
+        torch.cuda.synchronize()
+
+        def host_step(buffers):
+            """One end-to-end step, timed on the device: from the first copy-in (stream 0) to the
+            last copy-out (stream 2)."""
+            torch.cuda.synchronize()
+            e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e_a.record(streams[0])
+            shape.state.outer_step_host(variant, buffers, streams, args.chunk)
+            e_b.record(streams[2])
+            e_b.synchronize()
+            return e_a.elapsed_time(e_b)
+
+        def leg_bytes(k):
+            rows = 1 if k == "delta_prev_avg" else M
+            return rows * P * pinned[k].element_size()
+
+        per = [host_step(host) for _ in range(2 + n_steps)][2:]
+        e_ms = sum(per) / len(per)
+        if world > 1:
+            t = torch.tensor([e_ms], device=red_dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t[0])
+        used = [k for k in keys if pinned[k] is not None and not (k == "delta_prev_local" and variant != 2)
+                and not (k == "delta_prev_avg" and variant == 0)]
+        h2d = sum(leg_bytes(k) for k in used if not (k == "theta" and w.theta_kind == 2))
+        d2h = sum(leg_bytes(k) for k in used)
+        e2e = {"value": P * world / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "workload": shape.name, "M": M, "P_per_gpu": P, "ms_per_step": e_ms, "steps": len(per), "chunk": args.chunk,
+               "call": "diloco_outer_step_host: whole state in pinned host memory, copied in and out every step",
+               "timing": "CUDA events: first copy-in stream to last copy-out stream",
+               "pcie_GBps_each_way": h2d / e_ms / 1e6, "host_register_s": t_pin}
+        # second flavour: only theta crosses PCIe, the outer-optimiser state stays on the device
+        host_t = binding.make_buffers(theta=pinned["theta"], master=pinned["master"])
+        per = [host_step(host_t) for _ in range(2 + n_steps)][2:]
+        t_ms = sum(per) / len(per)
+        th_bytes = sum(leg_bytes(k) for k in ("theta", "master") if pinned[k] is not None)
+        e2e["theta_only"] = {"value": P * world / (t_ms * 1e-3), "ms_per_step": t_ms, "h2d_bytes_per_step":
+                             th_bytes if w.theta_kind != 2 else leg_bytes("master"), "d2h_bytes_per_step": th_bytes,
+                             "note": "theta travels, start / momentum / previous gradients resident on the device"}
+        torch.cuda.synchronize()
+        return e2e
+    except RuntimeError as ex:
+        return {"value": None, "unit": UNIT, "workload": shape.name, "error": str(ex)[:200]}
+    finally:
+        for t in pinned.values():
+            if t is not None:
+                try:
+                    unregister_host(torch, t)
+                except Exception:
+                    pass
+        pinned.clear()
+        gc.collect()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -239,90 +539,30 @@ def run_ours(args):
             dist.init_process_group("nccl", device_id=dev)
         else:
             dist.init_process_group(backend)
+    barrier = dist.barrier if world > 1 else None
+    peak, peak_kind = load_peak()
+    traffic = load_traffic()
     w = inputs.WORKLOADS[args.workload]
-    P = args.P or w.P                                       # per GPU: weak scaling, every rank the full shape
-    if args.strong:                                         # total work fixed: this rank's 64-aligned range
-        lo, hi = shard_bounds(P, world, rank)
-        P = hi - lo
-    variant = {"standard": 0, "delayed": 1, "eager": 2}[args.variant]
-    M = w.M
-    phase = w.H > 0 and not args.outer_only
-    th = {0: 4, 1: 2, 2: 6}[w.theta_kind]
-    need = M * P * (th + 12 + (8 + (2 if w.grad_kind else 4) if phase else 0)) + 4 * P + M * P * 4 + (512 << 20)
-    free = torch.cuda.mem_get_info(dev)[0]
-    if need > free:                                         # report, never run the device out of memory
+
+    main = Shape(args.workload, args, dev, rank, world, P=args.P or None, comm=args.comm)
+    ok, why = main.fits()
+    if world > 1:                                           # every rank must take the same branch
+        t = torch.tensor([0 if ok else 1], device=red_dev)
+        dist.all_reduce(t)
+        ok = int(t[0]) == 0
+    if not ok:                                              # report, never run the device out of memory
         if rank == 0:
             print(json.dumps({"metric": METRIC, "unit": UNIT, "value": None, "n_gpus": world,
-                              "config": {"workload": args.workload},
-                              "skipped": f"needs {need / 2**30:.1f} GiB of device memory, {free / 2**30:.1f} GiB free"}))
+                              "config": config_dict(args, w, main.P), "skipped": why}))
         return 0
-    st = inputs.make_outer_state(M, P, w.seed + 1000 * rank, device=dev, theta_kind=w.theta_kind, with_adam=phase)
-    stride = st["stride"]
-    state = binding.State.from_dict(st, H=w.H, outer_lr=w.outer_lr, outer_momentum=w.outer_momentum, beta1=w.beta1,
-                                    beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay, grad_kind=w.grad_kind,
-                                    impl=args.kernel)
-    grads = None
-    if phase:
-        if w.segments:
-            grads = torch.zeros((M, stride), dtype=torch.bfloat16 if w.grad_kind else torch.float32, device=dev)
-            inputs.make_segment_grads(M, inputs.segment_sizes(P, w.segments),
-                                      inputs.segment_scales(w.segments, st["gen"], dev).tolist(), st["gen"], grads)
-        else:
-            grads = inputs.make_grads(M, P, stride, st["gen"], dev, w.grad_kind)
+    sampler = ClockSampler(gpu)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    comm = {"f32": (0, 0, 0), "bf16": (1, 0, 0), "e4m3": (2, 4, 3), "e5m2": (2, 5, 2), "e2m1": (2, 2, 1),
-            "e3m0": (2, 3, 0)}[args.comm]
-    if comm[0]:
-        scratch = torch.zeros(64, dtype=torch.int32, device=dev)
-        state.close()
-        state = binding.State.from_dict(st, H=w.H, outer_lr=w.outer_lr, outer_momentum=w.outer_momentum, beta1=w.beta1,
-                                        beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay, grad_kind=w.grad_kind,
-                                        impl=args.kernel, comm_scratch=scratch)
-    run_outer = (lambda: state.outer_quantized(variant, *comm)) if comm[0] else (lambda: state.outer(variant))
-    outer_bpp = outer_bytes_per_param(variant, M, w.theta_kind)
-    if comm[0] == 2:                                    # the max-|Delta_m| pass re-reads theta and start
-        outer_bpp += M * ({0: 4, 1: 2, 2: 4}[w.theta_kind] + 4)
-    adam_bpp = adamw_bytes_per_param(M, w.theta_kind, w.grad_kind)
-
-    def one_step(timed):
-        """Returns (ms of the whole step, ms of the outer kernel alone)."""
-        if not phase:
-            inputs.inner_phase_standin(st)
-        flush.fill_(1)
-        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-        e0.record()
-        if phase:
-            for _ in range(w.H):
-                state.inner_adamw(grads, w.inner_lr)
-        e1.record()
-        run_outer()
-        e2.record()
-        if not timed:
-            return None
-        e2.synchronize()
-        return e0.elapsed_time(e2), e1.elapsed_time(e2), e0.elapsed_time(e1)
-
-    sampler = ClockSampler(gpu)                            # started before the warm-up: a short timed region
-    t_warm = time.perf_counter()                           # may see too few 100 ms samples of its own
-    for _ in range(args.warmup):
-        one_step(False)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    n0 = binding.launch_count()
-    t0 = time.perf_counter()
-    rows = [one_step(True) for _ in range(args.steps)]
-    torch.cuda.synchronize()
-    t1 = time.perf_counter()
-    launches = binding.launch_count() - n0
-    clocks = sampler.stop(t0, t1, t_warm)
-    if world > 1:
-        dist.barrier()
-    step_ms = sum(r[0] for r in rows) / len(rows)
-    outer_ms = sum(r[1] for r in rows) / len(rows)
-    outer_sorted = sorted(r[1] for r in rows)
-    outer_median, outer_min = outer_sorted[len(outer_sorted) // 2], outer_sorted[0]
-    adam_ms = sum(r[2] for r in rows) / len(rows) / max(1, w.H) if phase else None
+    main.allocate()
+    rows, launches, clocks = main.measure(flush, sampler, args.steps, args.warmup, barrier)
+    main_rec = main.record(rows, clocks, peak, traffic)
+    step_ms = main_rec["step_ms"]["mean"]
+    outer_ms = main_rec["outer"]["ms"]["mean"]
+    P, M, phase = main.P, w.M, main.phase
     if world > 1:
         t = torch.tensor([step_ms, outer_ms], device=red_dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -339,21 +579,26 @@ def run_ours(args):
     value = P_job / (step_ms * 1e-3)
 
     # --- roofline of the dominant kernel
-    peak, peak_kind = load_peak()
-    if phase and adam_ms * w.H > outer_ms:
-        dom, dom_ms, dom_bpp = "diloco_inner_adamw", adam_ms, adam_bpp
-    else:
-        dom, dom_ms, dom_bpp = f"diloco_outer_{args.variant}", outer_ms, outer_bpp
-    achieved = dom_bpp * P / (dom_ms * 1e-3) / 1e9
-    tr = None if comm[0] else NCU_TRAFFIC_BYTES_PER_PARAM.get((dom, M, w.theta_kind))
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                "algorithmic_bytes_per_param": dom_bpp, "traffic": (tr * P if tr else None),
-                "kernel_ms": dom_ms, "outer_ms_median": outer_median, "outer_ms_min": outer_min}
+    dom = main_rec["adamw"] if (phase and main_rec["adamw"]["ms"]["mean"] * w.H > outer_ms) else main_rec["outer"]
+    dom_ms = dom["ms"]["mean"] if dom is not main_rec["outer"] else outer_ms
+    achieved = dom["algorithmic_bytes_per_param"] * P / (dom_ms * 1e-3) / 1e9
+    tr = dom["ncu_dram_bytes_per_param"]
+    roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                "algorithmic_bytes_per_param": dom["algorithmic_bytes_per_param"], "traffic": (tr * P if tr else None),
+                "traffic_source": (f"ncu dram bytes per index of {dom['ncu_profile']} x P" if tr else None),
+                "kernel_ms": dom_ms, "outer_ms_median": main_rec["outer"]["ms"]["median"],
+                "outer_ms_min": main_rec["outer"]["ms"]["min"]}
+    if roofline["frac"] > 1.0:
+        roofline["frac_note"] = ("above 1: the denominator is a plain device copy (torch copy_), a reference point and "
+                                 "not a ceiling; see frac_of_nominal_8000 and copy_gbs_this_run")
 
-    # --- extra: the sibling kernels at the same shape (outer-only workloads, rank 0's GPU)
+    # --- extra: the sibling kernels at the same shape (outer-only workloads, explicit request)
     kernels = {}
     if args.siblings and not phase:
+        st = main.st
+        state, stride = main.state, st["stride"]
+
         def time_kernel(fn, n=5):
             ms = []
             for _ in range(2 + n):
@@ -364,7 +609,7 @@ def run_ours(args):
                 ms.append(a.elapsed_time(b))
             ms = ms[2:]
             return sum(ms) / len(ms)
-        for name, v in (("standard", 0), ("delayed", 1), ("eager", 2)):
+        for name, v in VARIANTS.items():
             ms = time_kernel(lambda v=v: state.outer(v))
             bpp = outer_bytes_per_param(v, M, w.theta_kind)
             kernels[f"outer_{name}"] = {"ms": ms, "GBps": bpp * P / ms / 1e6, "frac": bpp * P / ms / 1e6 / peak,
@@ -389,70 +634,95 @@ def run_ours(args):
                                       "params_per_s": P / ms * 1e3}
             sa.close(); del am, av, g
 
-    # --- end to end: state in pinned host memory, copies inside the timed region
-    e2e = None
-    if args.e2e and not phase and not comm[0]:
-        keys = ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom")
-        need = sum(st[k].numel() * st[k].element_size() for k in keys if st.get(k) is not None)
-        try:
-            pinned = {k: (torch.empty_like(st[k], device="cpu").pin_memory() if st.get(k) is not None else None) for k in keys}
-            for k in keys:
-                if pinned[k] is not None:
-                    pinned[k].copy_(st[k])
-            host = binding.make_buffers(**pinned)
-            streams = [torch.cuda.Stream(device=dev) for _ in range(3)]
-            torch.cuda.synchronize()
-            per = []
-            n_e2e = max(3, min(args.steps, 10))
-            def host_step(buffers):
-                """One end-to-end step, timed on the device: from the first copy-in (stream 0) to
-                the last copy-out (stream 2)."""
-                torch.cuda.synchronize()
-                e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e_a.record(streams[0])
-                state.outer_step_host(variant, buffers, streams, args.chunk)
-                e_b.record(streams[2])
-                e_b.synchronize()
-                return e_a.elapsed_time(e_b)
+    # --- end to end: state in pinned host memory, copies inside the timed region.  On the main
+    # workload if its state may be page-locked (a fraction of the host's available memory, shared
+    # by the ranks of this node), else on the largest other eager shape that may, and says which.
+    e2e, e2e_shape = None, None
+    if args.e2e and not phase and not main.comm[0]:
+        budget = mem_available_bytes() * args.e2e_host_fraction / max(1, int(os.environ.get("LOCAL_WORLD_SIZE", world)))
+        order = [args.workload] + [n for n in ("cfg4a", "cfg4b", "cfg4c", "cfg1", "cfg0") if n != args.workload]
+        if args.P:
+            order = [args.workload]
+        pick = None
+        for n in order:
+            Pn = main.P if n == args.workload else inputs.WORKLOADS[n].P
+            wn = inputs.WORKLOADS[n]
+            if wn.H == 0 and state_bytes_per_param(wn.M, wn.theta_kind) * Pn <= budget:
+                pick = n
+                break
+        if pick == args.workload:
+            e2e = run_e2e(main, args, world, dist, red_dev, max(3, min(args.steps, 10 if main.P < 2e8 else 3)))
+        elif pick is not None:
+            e2e_shape = pick                                   # measured below, once the main state is freed
+        else:
+            e2e = {"value": None, "unit": UNIT, "error": f"no shape fits {budget / 2**30:.0f} GiB of pinned host memory"}
+    main.free()
+    if e2e_shape is not None:
+        sh = Shape(e2e_shape, args, dev, rank, world)
+        ok, why = sh.fits()
+        if ok:
+            sh.allocate()
+            e2e = run_e2e(sh, args, world, dist, red_dev, 3)
+            e2e["note"] = (f"{args.workload}'s state exceeds the pinned-memory budget of this host; measured on "
+                           f"{e2e_shape}, the largest eager shape that fits")
+        else:
+            e2e = {"value": None, "unit": UNIT, "workload": e2e_shape, "error": why}
+        sh.free()
 
-            for i in range(2 + n_e2e):
-                per.append(host_step(host))
-            per = per[2:]
-            e_ms = sum(per) / len(per)
-            if world > 1:
-                t = torch.tensor([e_ms], device=red_dev, dtype=torch.float64)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                e_ms = float(t[0])
-            def leg_bytes(k):
-                rows = 1 if k == "delta_prev_avg" else M
-                return rows * P * pinned[k].element_size()
-            used = [k for k in keys if pinned[k] is not None and not (k == "delta_prev_local" and variant != 2)
-                    and not (k == "delta_prev_avg" and variant == 0)]
-            h2d = sum(leg_bytes(k) for k in used if not (k == "theta" and w.theta_kind == 2))
-            d2h = sum(leg_bytes(k) for k in used)
-            e2e = {"value": P_job / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                   "ms_per_step": e_ms, "chunk": args.chunk, "timing": "CUDA events: first copy-in stream to last copy-out stream",
-                   "pcie_GBps_each_way": h2d / e_ms / 1e6}
-            # second flavour: only theta crosses PCIe, the outer-optimiser state stays on the device
-            host_t = binding.make_buffers(theta=pinned["theta"], master=pinned["master"])
-            per = []
-            for i in range(2 + n_e2e):
-                per.append(host_step(host_t))
-            t_ms = sum(per[2:]) / len(per[2:])
-            th_bytes = sum(leg_bytes(k) for k in ("theta", "master") if pinned[k] is not None)
-            e2e["theta_only"] = {"value": P_job / (t_ms * 1e-3), "ms_per_step": t_ms, "h2d_bytes_per_step":
-                                 th_bytes if w.theta_kind != 2 else leg_bytes("master"), "d2h_bytes_per_step": th_bytes,
-                                 "note": "theta travels, start / momentum / previous gradients resident on the device"}
-            del pinned
-        except RuntimeError as ex:
-            e2e = {"value": None, "unit": UNIT, "error": str(ex)[:200]}
+    # --- the other headline shapes, each measured like the main one, with its own clock record
+    shapes = {}
+    if args.shapes and world == 1 and not args.P:
+        shapes[args.workload] = main_rec
+        plan = [("cfg1", None, 10), ("cfg4a", None, 10), ("cfg4b", None, 10), ("cfg4c", None, 10),
+                ("cfg2", True, 3), ("cfg3", True, 3)]
+        for name, ph, n in plan:
+            if name == args.workload and ph is None:
+                continue
+            sh = Shape(name, args, dev, rank, world, phase=ph, variant=2)
+            ok, why = sh.fits()
+            if not ok:
+                shapes[name] = {"skipped": why}
+                continue
+            try:
+                sh.allocate()
+                r, _, c = sh.measure(flush, sampler, min(args.steps, n), 3)
+                shapes[name] = sh.record(r, c, peak, traffic)
+            except RuntimeError as ex:                          # e.g. an allocation that fails after the pre-check
+                shapes[name] = {"skipped": str(ex)[:200]}
+            sh.free()
+        # cfg0: 37.7 MB of state, smaller than L2.  Cold = as everywhere (replicas moved, L2 flushed
+        # before each step); warm = the same launches back to back on an L2-resident state.
+        sh = Shape("cfg0", args, dev, rank, world, variant=2).allocate()
+        r, _, c = sh.measure(flush, sampler, 20, 3)
+        cold = sh.record(r, c, peak, traffic)
+        r, _, c = sh.measure(flush, sampler, 50, 5, move=False, do_flush=False)
+        warm = sh.record(r, c, peak, traffic)
+        shapes["cfg0"] = dict(cold, l2="cold: L2 flushed before every step",
+                              warm_l2={"outer": warm["outer"], "clocks": warm["clocks"],
+                                       "l2": "warm: back-to-back launches, state resident in L2; GB/s is not HBM bandwidth"})
+        sh.free()
+
+    # --- a plain device copy measured in this run, the same way the recorded peak was
+    copy_gbs = None
+    if world == 1:
+        n = 1 << 30
+        if torch.cuda.mem_get_info(dev)[0] > 6 * n:
+            a = torch.empty(n, dtype=torch.bfloat16, device=dev); b = torch.empty_like(a)
+            a.fill_(1)
+            best = 1e9
+            for _ in range(10):
+                x, y = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                x.record(); b.copy_(a); y.record(); y.synchronize()
+                best = min(best, x.elapsed_time(y))
+            copy_gbs = 2 * 2 * n / best / 1e6
+            del a, b
 
     # --- CPU baseline: the oracle as it stands, bounded sample, rank 0 at N = 1 only
     cpu = None
     if args.cpu_baseline and world == 1:
         import oracle
         oracle.build()
-        Ps = min(P, 35_000_000)
+        Ps = oracle_sample_size(w, P)
         _, h = host_state(w, Ps, w.seed)
         cores = os.cpu_count() or 1
         s_stride = inputs.padded_stride(Ps)
@@ -460,25 +730,19 @@ def run_ours(args):
         tm = time_oracle_eager(h, M, Ps, s_stride, w.theta_kind, w.outer_lr, w.outer_momentum, cores, 8.0)
         t1c = time_oracle_eager(h, M, Ps, s_stride, w.theta_kind, w.outer_lr, w.outer_momentum, 1, 4.0)
         cpu = {"value": Ps / (sum(tm) / len(tm)), "unit": UNIT, "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
-               "sample": f"eager outer step on M={M}, P={Ps} of {P} (all replicas, drawn on the host with the same recipe), "
-                         f"{len(tm)} steps with {cores} OpenMP threads",
+               "sample": f"eager outer step on the first {Ps} of {P} parameters of all {M} replicas (drawn on the host "
+                         f"with the same recipe), {len(tm)} steps with {cores} OpenMP threads",
                "single_thread_value": Ps / (sum(t1c) / len(t1c))}
+    sampler.stop()
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": step_ms, "higher_is_better": True, "scaling": "strong" if args.strong else "weak", "vs_baseline": None,
-                "dtype": "f32", "data": "synthetic",
-                "config": {"workload": args.workload, "variant": args.variant, "M": M, "P_per_gpu": P,
-                           "theta": ["f32", "bf16", "f32 master + bf16 copy"][w.theta_kind],
-                           "step": (f"{w.H} x inner AdamW + 1 outer {args.variant}" if phase else f"1 outer {args.variant} step"),
-                           "outer_lr": w.outer_lr, "outer_momentum": w.outer_momentum,
-                           "l2": "state >> 126 MB L2 and a 256 MB flush write between steps",
-                           "sharding": "parameter axis split across ranks, all M replicas of an index on one rank, no collective",
-                           "kernel_impl": ["auto", "direct", "bulk"][args.kernel], "outer_gradient_wire_format": args.comm},
+                "dtype": "f32", "data": "synthetic", "config": config_dict(args, w, P),
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
-                "replica_params_per_s": value * M, "kernels": kernels or None}
+                "replica_params_per_s": value * M, "copy_gbs_this_run": copy_gbs, "kernels": kernels or None,
+                "shapes": shapes or None}
         print(json.dumps(line))
-    state.close()
     if world > 1:
         dist.destroy_process_group()
     return 0
@@ -494,7 +758,7 @@ def report(args):
         if w.H:
             runs = [runs[0] + ["--steps", "3"], runs[0] + ["--outer-only"]]
         for extra in runs:
-            cmd = [sys.executable, str(ROOT / "bench.py"), "--no-e2e", "--no-cpu-baseline"] + extra
+            cmd = [sys.executable, str(ROOT / "bench.py"), "--no-e2e", "--no-cpu-baseline", "--no-shapes", "--siblings"] + extra
             out = subprocess.run(cmd, capture_output=True, text=True)
             line = [l for l in out.stdout.splitlines() if l.startswith("{")]
             if out.returncode != 0 or not line:
@@ -523,17 +787,22 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1")
-    ap.add_argument("--variant", default="eager", choices=["standard", "delayed", "eager"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--variant", default="eager", choices=list(VARIANTS))
     ap.add_argument("--P", type=int, default=0, help="override the workload's parameter count (per GPU)")
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 direct, 2 bulk")
-    ap.add_argument("--comm", default="f32", choices=["f32", "bf16", "e4m3", "e5m2", "e2m1", "e3m0"],
+    ap.add_argument("--comm", default="f32", choices=list(COMM),
                     help="wire format of the outer gradients (quantised communication)")
     ap.add_argument("--chunk", type=int, default=64 * 16384, help="elements per chunk of the host-buffer path")
+    ap.add_argument("--e2e-host-fraction", type=float, default=0.5,
+                    help="share of the host's available memory that the end-to-end leg may page-lock")
     ap.add_argument("--strong", action="store_true", help="split the workload's P across ranks instead of one full shape per rank")
     ap.add_argument("--outer-only", action="store_true", help="phase workloads: time the outer step alone")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--no-shapes", dest="shapes", action="store_false",
+                    help="skip the record of the other headline shapes (single-GPU default run)")
+    ap.add_argument("--siblings", action="store_true", help="also time the sibling kernels at the main shape")
     ap.add_argument("--no-siblings", dest="siblings", action="store_false")
     ap.add_argument("--report", action="store_true",
                     help="run every workload (one process each) and print a table of all kernels to stderr")

@@ -83,7 +83,11 @@ enum {
 enum {
   DILOCO_IMPL_AUTO = 0,
   DILOCO_IMPL_DIRECT = 1, /* register-resident columns, 128-bit global loads and stores */
-  DILOCO_IMPL_BULK = 2    /* replica tiles staged through shared memory by the TMA unit (1-D bulk copies) */
+  DILOCO_IMPL_BULK = 2,   /* replica tiles staged through shared memory by the TMA unit (1-D bulk copies) */
+  /* force one of the warp-split forms (replica axis over the warps of a block) whatever M is,
+     for measurements; AUTO picks among them and the per-M shapes by M */
+  DILOCO_IMPL_SPLIT_R2 = 3, /* two replicas per warp, 128-bit accesses (M <= 32, else as AUTO) */
+  DILOCO_IMPL_SPLIT_R4 = 4  /* four replicas per warp, 64-bit accesses                          */
 };
 
 typedef struct {

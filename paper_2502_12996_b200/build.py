@@ -10,8 +10,8 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libdiloco.so"
 REPORT = PKG / "ptxas_report.txt"        # registers / spills of every kernel, written by each build
-OUTER_M = [0, 1, 2, 3, 4, 8, 1000, 1001]    # translation units: replica counts with kernels of their own, and
-                                            # the run-time forms (0 two-sweep, 1000 warp split, 1001 warp per replica)
+OUTER_M = [0, 1, 2, 3, 4, 8, 1000, 1002]   # translation units: replica counts with kernels of their own, the
+                                                 # warp-split forms (1000, 1002) and the first-steps form (0)
 OBJ = PKG / "_obj"
 
 NVCC_FLAGS = [

@@ -21,11 +21,11 @@
 
 using namespace diloco;
 
-// launch_outer_shape<M, Q> is instantiated in diloco_outer_m.cu, once per replica count
-#define DILOCO_EXTERN(M_)                                                                                       \
-  extern template int diloco::launch_outer_shape<M_, false>(int, int, bool, const OuterArgs &, cudaStream_t); \
-  extern template int diloco::launch_outer_shape<M_, true>(int, int, bool, const OuterArgs &, cudaStream_t);
-DILOCO_FOR_EACH_M(DILOCO_EXTERN)
+// launch_outer_shape<ID, Q> is instantiated in diloco_outer_m.cu, once per shape
+#define DILOCO_EXTERN(ID_)                                                                                 \
+  extern template int diloco::launch_outer_shape<ID_, false>(int, int, const OuterArgs &, cudaStream_t); \
+  extern template int diloco::launch_outer_shape<ID_, true>(int, int, const OuterArgs &, cudaStream_t);
+DILOCO_FOR_EACH_SHAPE(DILOCO_EXTERN)
 #undef DILOCO_EXTERN
 
 // One fragment of the parameter axis with its own outer-step schedule (Streaming DiLoCo applies
@@ -80,7 +80,7 @@ int validate_config(const diloco_config_t *c) {
   if (c->M > DILOCO_MAX_M) return DILOCO_ERR_UNSUPPORTED;
   if (c->theta_kind < DILOCO_THETA_F32 || c->theta_kind > DILOCO_THETA_MASTER_BF16) return DILOCO_ERR_INVALID_ARG;
   if (c->grad_kind < DILOCO_GRAD_F32 || c->grad_kind > DILOCO_GRAD_BF16) return DILOCO_ERR_INVALID_ARG;
-  if (c->impl < DILOCO_IMPL_AUTO || c->impl > DILOCO_IMPL_BULK) return DILOCO_ERR_INVALID_ARG;
+  if (c->impl < DILOCO_IMPL_AUTO || c->impl > DILOCO_IMPL_SPLIT_R4) return DILOCO_ERR_INVALID_ARG;
   if (!(c->outer_momentum >= 0.f && c->outer_momentum < 1.f)) return DILOCO_ERR_INVALID_ARG;
   if (!std::isfinite(c->outer_lr)) return DILOCO_ERR_INVALID_ARG;
   if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f)) return DILOCO_ERR_INVALID_ARG;
@@ -122,20 +122,33 @@ int validate_buffers(const diloco_config_t *c, const diloco_buffers_t *b) {
   return DILOCO_OK;
 }
 
+// Which warp-split form serves a replica count that has no compile-time shape (see
+// diloco_outer_launch.cuh); `forced` (a state's impl field, for measurements) overrides it.
+int split_shape_for(int M, int forced) {
+  if (forced == DILOCO_IMPL_SPLIT_R2 && M <= 32) return SHAPE_SPLIT_R2; // 16 warps per block at most
+  if (forced == DILOCO_IMPL_SPLIT_R4) return SHAPE_SPLIT_R4;
+  return M <= 20 ? SHAPE_SPLIT_R2 : SHAPE_SPLIT_R4;
+}
+
 template <bool Q>
 int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterArgs &a, cudaStream_t s) {
-  const int tk = st->cfg.theta_kind, M = st->cfg.M;
-  switch (M) {
-    case 1: return launch_outer_shape<1, Q>(var, tk, boot, a, s);
-    case 2: return launch_outer_shape<2, Q>(var, tk, boot, a, s);
-    case 3: return launch_outer_shape<3, Q>(var, tk, boot, a, s);
-    case 4: return launch_outer_shape<4, Q>(var, tk, boot, a, s);
-    case 8: return launch_outer_shape<8, Q>(var, tk, boot, a, s);
-    default: break;
+  const int tk = st->cfg.theta_kind, M = st->cfg.M, impl = st->cfg.impl;
+  if (boot) return launch_outer_shape<SHAPE_FIRST_STEPS, Q>(var, tk, a, s);
+  const bool forced_split = impl == DILOCO_IMPL_SPLIT_R2 || impl == DILOCO_IMPL_SPLIT_R4;
+  if (!forced_split) {
+    switch (M) {
+      case 1: return launch_outer_shape<1, Q>(var, tk, a, s);
+      case 2: return launch_outer_shape<2, Q>(var, tk, a, s);
+      case 3: return launch_outer_shape<3, Q>(var, tk, a, s);
+      case 4: return launch_outer_shape<4, Q>(var, tk, a, s);
+      case 8: return launch_outer_shape<8, Q>(var, tk, a, s);
+      default: break;
+    }
   }
-  if (M % 4 == 0) return launch_outer_shape<SHAPE_WARP_SPLIT, Q>(var, tk, boot, a, s);       // 12, 16, ..., 64
-  if (M <= 7) return launch_outer_shape<SHAPE_WARP_PER_REPLICA, Q>(var, tk, boot, a, s);     // 5, 6, 7
-  return launch_outer_shape<SHAPE_TWO_SWEEP, Q>(var, tk, boot, a, s);
+  switch (split_shape_for(M, impl)) {
+    case SHAPE_SPLIT_R2: return launch_outer_shape<SHAPE_SPLIT_R2, Q>(var, tk, a, s);
+    default: return launch_outer_shape<SHAPE_SPLIT_R4, Q>(var, tk, a, s);
+  }
 }
 
 // Delayed and eager steps consume the gradients recorded overlap_steps outer steps ago: the
@@ -258,19 +271,9 @@ int launch_bulk_t(const diloco_state *st, const OuterArgs &a, cudaStream_t s) {
 
 template <int M, int T, int S, int NT>
 int launch_bulk_m(const diloco_state *st, int var, int tk, const OuterArgs &a, cudaStream_t s) {
-#define DILOCO_CASE(VAR_, TK_) \
-  if (var == VAR_ && tk == TK_) return launch_bulk_t<M, VAR_, TK_, T, S, NT>(st, a, s);
-  DILOCO_CASE(VAR_STANDARD, TK_F32)
-  DILOCO_CASE(VAR_STANDARD, TK_BF16)
-  DILOCO_CASE(VAR_STANDARD, TK_MASTER_BF16)
-  DILOCO_CASE(VAR_DELAYED, TK_F32)
-  DILOCO_CASE(VAR_DELAYED, TK_BF16)
-  DILOCO_CASE(VAR_DELAYED, TK_MASTER_BF16)
-  DILOCO_CASE(VAR_EAGER, TK_F32)
-  DILOCO_CASE(VAR_EAGER, TK_BF16)
-  DILOCO_CASE(VAR_EAGER, TK_MASTER_BF16)
-#undef DILOCO_CASE
-  return DILOCO_ERR_INVALID_ARG;
+  return dispatch_variant_storage(var, tk, [&](auto var_, auto tk_) {
+    return launch_bulk_t<M, decltype(var_)::value, decltype(tk_)::value, T, S, NT>(st, a, s);
+  });
 }
 
 int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t len, cudaStream_t s, int ring = -1) {
@@ -870,7 +873,7 @@ int diloco_set_outer_hparams(diloco_state_t *st, float outer_lr, float outer_mom
 }
 
 int diloco_set_impl(diloco_state_t *st, int32_t impl) {
-  if (!st || impl < DILOCO_IMPL_AUTO || impl > DILOCO_IMPL_BULK) return DILOCO_ERR_INVALID_ARG;
+  if (!st || impl < DILOCO_IMPL_AUTO || impl > DILOCO_IMPL_SPLIT_R4) return DILOCO_ERR_INVALID_ARG;
   st->cfg.impl = impl;
   return DILOCO_OK;
 }

@@ -270,7 +270,7 @@ __global__ void __launch_bounds__(NT, 1) outer_step_bulk_kernel(const OuterArgs 
   if (blockIdx.x == gridDim.x - 1 && !aborted) {
     const long long done = ntiles * T;
     const long long nvec = (a.P - done) / 4;
-    for (long long j = tid; j < nvec; j += NT) outer_column<M, 1, VAR, TK, false, 4>(a, done + j * 4, 0, true);
+    for (long long j = tid; j < nvec; j += NT) outer_column<M, 1, VAR, TK, 4>(a, done + j * 4, 0, true);
     for (long long i = done + nvec * 4 + tid; i < a.P; i += NT) outer_column_rt<VAR, TK, false, 1>(a, i);
   }
 }

@@ -295,8 +295,10 @@ __global__ void __launch_bounds__(NT) delta_amax_kernel(const OuterArgs a, unsig
 // lanes apart in one warp and pass the running sum of the local outer gradients from group
 // to group with shuffles, so the mean is still the left-to-right sum m = 0 .. M-1 and every
 // lane divides the same total (identical bits in all G lanes).  Splitting the replica axis
-// keeps the per-thread register count of M = 8 .. 64 at that of M = 4.
-template <int R, int G, int VAR, int TK, bool BOOT, int V, bool Q = false>
+// keeps the per-thread register count of M = 8 at that of M = 4.
+// (The first outer steps of a delayed / eager run, which only record, go through
+// outer_column_rt<BOOT = true> for every M: they happen once per run.)
+template <int R, int G, int VAR, int TK, int V, bool Q = false>
 __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, int m0, bool active) {
   constexpr int CW = 32 / G;
   float s[R][V], d[R][V], b[R][V], pl[R][V], pa[V], mean[V];
@@ -308,26 +310,20 @@ __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, in
       const long long at = (m0 + r) * a.stride + i;
       F32Vec<V>::load(a.start + at, s[r]);
       load_theta<TK, V>(a, at, d[r]);
-      if (!BOOT) {
-        F32Vec<V>::load(a.mom + at, b[r]);
-        if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + at, pl[r]);
-      }
+      F32Vec<V>::load(a.mom + at, b[r]);
+      if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + at, pl[r]);
     }
-    if (!BOOT && VAR != VAR_STANDARD) F32Vec<V>::load(a.dpa + i, pa);
+    if (VAR != VAR_STANDARD) F32Vec<V>::load(a.dpa + i, pa);
   } else {
 #pragma unroll
     for (int r = 0; r < R; ++r)
 #pragma unroll
       for (int e = 0; e < V; ++e) s[r][e] = d[r][e] = 0.f;
   }
-  float x[R][V]; // theta_m^(t), needed again by the first outer step
 #pragma unroll
   for (int r = 0; r < R; ++r)
 #pragma unroll
-    for (int e = 0; e < V; ++e) {
-      x[r][e] = d[r][e];
-      d[r][e] = s[r][e] - d[r][e]; // line 7: Delta_m
-    }
+    for (int e = 0; e < V; ++e) d[r][e] = s[r][e] - d[r][e]; // line 7: Delta_m
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const float scale = Q ? comm_scale(a, m0 + r) : 1.f;
@@ -365,17 +361,6 @@ __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, in
 #pragma unroll
   for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
   if (!active) return;
-
-  if constexpr (BOOT) {
-    // first outer step (t = H): record the gradients, restart from the current parameters
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const long long at = (m0 + r) * a.stride + i;
-      F32Vec<V>::store(a.start + at, x[r]);
-      if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d[r]);
-    }
-    if (m0 == 0) F32Vec<V>::store(a.dpa + i, mean);
-  } else {
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     const long long at = (m0 + r) * a.stride + i;
@@ -399,7 +384,6 @@ __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, in
     if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d[r]);
   }
   if (VAR != VAR_STANDARD && m0 == 0) F32Vec<V>::store(a.dpa + i, mean);
-  }
 }
 
 // ---------------------------------------------------------------- outer step, runtime M
@@ -462,78 +446,90 @@ __device__ __forceinline__ void outer_column_rt(const OuterArgs &a, long long i)
 
 // One column per thread (per G lanes), one launch wave after the other: the hardware block
 // scheduler refills an SM as soon as a CTA retires, which measured ~10 % faster than a
-// persistent grid-stride loop.  M = 0 selects the runtime-M form (G = 1).
+// persistent grid-stride loop.
 // Grid: ceil(ceil(nvec / CW) * 32 / NT) blocks, nvec = P / V, CW = 32 / G.  The ragged tail
 // (P % V indices) is done one index per thread by the last block with the runtime-M code.
-template <int M, int G, int VAR, int TK, bool BOOT, int V, int NT, int MINB, bool Q = false>
+template <int M, int G, int VAR, int TK, int V, int NT, int MINB, bool Q = false>
 __global__ void __launch_bounds__(NT, MINB) outer_step_kernel(const OuterArgs a) {
+  static_assert(M >= 1 && M % G == 0, "replicas must divide evenly over the lane groups");
   constexpr int CW = 32 / G;
+  constexpr int R = M / G;
   const long long nvec = a.P / V;
   const long long t = (long long)blockIdx.x * NT + threadIdx.x;
   const int lane = threadIdx.x & 31;
   const long long j = (t >> 5) * CW + (lane % CW);
-  if (M > 0) {
-    constexpr int R = (M > 0 ? M : 1) / G;
-    const bool active = j < nvec;
-    if (G > 1 || active) outer_column<R, G, VAR, TK, BOOT, V, Q>(a, j * V, (lane / CW) * R, active);
-  } else {
-    if (j < nvec) outer_column_rt<VAR, TK, BOOT, V, Q>(a, j * V);
-  }
+  const bool active = j < nvec;
+  if (G > 1 || active) outer_column<R, G, VAR, TK, V, Q>(a, j * V, (lane / CW) * R, active);
   if (blockIdx.x == gridDim.x - 1) {
     const long long i = nvec * V + threadIdx.x;
-    if (i < a.P) outer_column_rt<VAR, TK, BOOT, 1, Q>(a, i);
+    if (i < a.P) outer_column_rt<VAR, TK, false, 1, Q>(a, i);
   }
 }
 
-// ---------------------------------------------------------------- outer step, many replicas
-// Large M does not fit the lane split: 8 or 16 lanes per column would leave 64- or 32-byte
-// runs per row.  Here the replica axis is split across the WARPS of a block instead: warp w owns
-// replicas 4w .. 4w+3 of 32 columns (32 V-element vectors per row and access), every warp
-// leaves what its replicas send (Delta_m, or its wire rounding) in shared memory, and after
-// one barrier every thread sums all M contributions of its own 4 indices in the order
-// m = 0 .. M-1: the same left-to-right sum as everywhere else.  Block = M/4 warps; M is a
-// run-time multiple of 4 (12 .. 64), so one set of kernels serves all of them.
-template <int VAR, int TK, bool BOOT, bool Q, int V>
-__global__ void __launch_bounds__(512, 2) outer_step_cta_kernel(const OuterArgs a) {
-  constexpr int R = 4;                 // a.M is a multiple of 4, at most 64: block = 8 M threads
+// The first outer steps of a delayed / eager run (t <= D H: record the gradients, restart from
+// the current parameters, apply nothing), any M at run time, one column per thread.  They run
+// once per training run, so one plain form serves every replica count.
+template <int VAR, int TK, int V, int NT, bool Q = false>
+__global__ void __launch_bounds__(NT, 4) outer_first_steps_kernel(const OuterArgs a) {
+  const long long nvec = a.P / V;
+  const long long j = (long long)blockIdx.x * NT + threadIdx.x;
+  if (j < nvec) outer_column_rt<VAR, TK, true, V, Q>(a, j * V);
+  if (blockIdx.x == gridDim.x - 1) {
+    const long long i = nvec * V + threadIdx.x;
+    if (i < a.P) outer_column_rt<VAR, TK, true, 1, Q>(a, i);
+  }
+}
+
+// ---------------------------------------------------------------- outer step, replica axis over warps
+// Replica counts that have no compile-time shape (5, 6, 7 and everything from 9 to 64; M is a
+// run-time argument).  A lane split would leave runs of 64 bytes or less per row and access
+// here; instead the replica axis is split across the WARPS of a block: warp w owns replicas
+// w R .. w R + R - 1 (the last warp possibly fewer) of 32 columns of V indices, so every row is
+// still read and written 32 V elements at a time.  Every warp leaves what its replicas send
+// (Delta_m, or its wire rounding) in shared memory, and after one barrier every thread sums
+// all M contributions of its own V indices in the order m = 0 .. M-1: the same left-to-right
+// sum as everywhere else.  Block = ceil(M / R) warps, shared memory M x V x 32 floats.
+template <int VAR, int TK, bool Q, int V, int R>
+__global__ void __launch_bounds__(512, 2) outer_step_split_kernel(const OuterArgs a) {
   extern __shared__ float sent_dyn[];  // [M][V][32]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int m0 = warp * R;
+  const int mine = min(R, a.M - m0);   // replicas of this warp: R, fewer in the last warp
   const long long nvec = a.P / V;
   const long long j = (long long)blockIdx.x * 32 + lane;
   const bool active = j < nvec;
   const long long i = j * V;
-  float s[R][V], d[R][V], b[R][V], pl[R][V], pa[V], x[R][V], mean[V];
-  if (active) {
+  float s[R][V], d[R][V], b[R][V], pl[R][V], pa[V], mean[V];
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
+  for (int r = 0; r < R; ++r) {
+    if (active && r < mine) {
       const long long at = (m0 + r) * a.stride + i;
       F32Vec<V>::load(a.start + at, s[r]);
       load_theta<TK, V>(a, at, d[r]);
-      if (!BOOT) {
-        F32Vec<V>::load(a.mom + at, b[r]);
-        if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + at, pl[r]);
-      }
+      F32Vec<V>::load(a.mom + at, b[r]);
+      if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + at, pl[r]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < V; ++e) s[r][e] = d[r][e] = b[r][e] = pl[r][e] = 0.f;
     }
-    if (!BOOT && VAR != VAR_STANDARD) F32Vec<V>::load(a.dpa + i, pa);
-  } else {
+  }
+  if (VAR != VAR_STANDARD) {
+    if (active) F32Vec<V>::load(a.dpa + i, pa);
+    else {
 #pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-      for (int e = 0; e < V; ++e) s[r][e] = d[r][e] = 0.f;
+      for (int e = 0; e < V; ++e) pa[e] = 0.f;
+    }
   }
 #pragma unroll
   for (int r = 0; r < R; ++r) {
-    const float scale = Q ? comm_scale(a, m0 + r) : 1.f;
-    float w[V];
+    if (r < mine) {
+      const float scale = Q ? comm_scale(a, m0 + r) : 1.f;
 #pragma unroll
-    for (int e = 0; e < V; ++e) {
-      x[r][e] = d[r][e];
-      d[r][e] = s[r][e] - d[r][e];                                  // Alg. 1-3 line 7
-      w[e] = Q ? comm_round(d[r][e], scale, a) : d[r][e];
+      for (int e = 0; e < V; ++e) {
+        d[r][e] = s[r][e] - d[r][e];                                  // Alg. 1-3 line 7
+        sent_dyn[((m0 + r) * V + e) * 32 + lane] = Q ? comm_round(d[r][e], scale, a) : d[r][e];
+      }
     }
-#pragma unroll
-    for (int e = 0; e < V; ++e) sent_dyn[((m0 + r) * V + e) * 32 + lane] = w[e];
   }
   __syncthreads();
   // line 8: Delta = (1/M) sum_m (what replica m sent), m in order
@@ -548,17 +544,9 @@ __global__ void __launch_bounds__(512, 2) outer_step_cta_kernel(const OuterArgs 
 #pragma unroll
   for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
   if (active) {
-    if constexpr (BOOT) {
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const long long at = (m0 + r) * a.stride + i;
-        F32Vec<V>::store(a.start + at, x[r]);
-        if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d[r]);
-      }
-      if (warp == 0) F32Vec<V>::store(a.dpa + i, mean);
-    } else {
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
+    for (int r = 0; r < R; ++r) {
+      if (r < mine) {
         const long long at = (m0 + r) * a.stride + i;
 #pragma unroll
         for (int e = 0; e < V; ++e) {
@@ -577,87 +565,12 @@ __global__ void __launch_bounds__(512, 2) outer_step_cta_kernel(const OuterArgs 
         store_theta<TK, V>(a, at, s[r]);
         if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d[r]);
       }
-      if (VAR != VAR_STANDARD && warp == 0) F32Vec<V>::store(a.dpa + i, mean);
     }
+    if (VAR != VAR_STANDARD && warp == 0) F32Vec<V>::store(a.dpa + i, mean);
   }
   if (blockIdx.x == gridDim.x - 1) { // ragged tail, one index per thread
     const long long t = nvec * V + threadIdx.x;
-    if (t < a.P) outer_column_rt<VAR, TK, BOOT, 1, Q>(a, t);
-  }
-}
-
-// ---------------------------------------------------------------- outer step, small odd M
-// One warp per replica, M <= 8 chosen at launch (block = 32 M threads, shared memory M x V x 32
-// floats): warp m owns replica m of 32 columns, leaves what it sends in shared memory, and
-// after one barrier every thread forms the ordered sum m = 0 .. M-1 for its own indices.
-// Serves the small replica counts that have no compile-time shape (5, 6, 7); with more warps
-// per block the barrier costs more than it saves (M = 12: 5.0 TB/s, M = 24: 3.4).
-template <int VAR, int TK, bool BOOT, bool Q, int V>
-__global__ void __launch_bounds__(256, 4) outer_step_warp_per_replica_kernel(const OuterArgs a) {
-  extern __shared__ float sent_dyn[]; // [M][V][32]
-  const int lane = threadIdx.x & 31, m = threadIdx.x >> 5;
-  const long long nvec = a.P / V;
-  const long long j = (long long)blockIdx.x * 32 + lane;
-  const bool active = j < nvec;
-  const long long i = j * V, at = m * a.stride + i;
-  float s[V], d[V], b[V], pl[V], pa[V], x[V], mean[V];
-  if (active) {
-    F32Vec<V>::load(a.start + at, s);
-    load_theta<TK, V>(a, at, d);
-    if (!BOOT) {
-      F32Vec<V>::load(a.mom + at, b);
-      if (VAR == VAR_EAGER) F32Vec<V>::load(a.dpl + at, pl);
-      if (VAR != VAR_STANDARD) F32Vec<V>::load(a.dpa + i, pa);
-    }
-  } else {
-#pragma unroll
-    for (int e = 0; e < V; ++e) s[e] = d[e] = 0.f;
-  }
-  const float scale = Q ? comm_scale(a, m) : 1.f;
-#pragma unroll
-  for (int e = 0; e < V; ++e) {
-    x[e] = d[e];
-    d[e] = s[e] - d[e];                                             // Alg. 1-3 line 7
-    sent_dyn[(m * V + e) * 32 + lane] = Q ? comm_round(d[e], scale, a) : d[e];
-  }
-  __syncthreads();
-  for (int q = 0; q < a.M; ++q) {                                   // line 8, replica order
-#pragma unroll
-    for (int e = 0; e < V; ++e) {
-      const float w = sent_dyn[(q * V + e) * 32 + lane];
-      mean[e] = (q == 0) ? w : mean[e] + w;
-    }
-  }
-#pragma unroll
-  for (int e = 0; e < V; ++e) mean[e] = mean[e] / a.fM;
-  if (active) {
-    if constexpr (BOOT) {
-      F32Vec<V>::store(a.start + at, x);
-      if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d);
-      if (m == 0) F32Vec<V>::store(a.dpa + i, mean);
-    } else {
-#pragma unroll
-      for (int e = 0; e < V; ++e) {
-        float g;
-        if (VAR == VAR_STANDARD) g = mean[e];
-        else if (VAR == VAR_DELAYED) g = pa[e];
-        else {
-          float t = d[e] - pl[e];                                    // Alg. 3 line 11
-          t = t / a.fM;
-          g = t + pa[e];
-        }
-        nesterov(g, a.eta, a.mu, b[e], s[e]);
-      }
-      F32Vec<V>::store(a.mom + at, b);
-      F32Vec<V>::store(a.start + at, s);
-      store_theta<TK, V>(a, at, s);
-      if (VAR == VAR_EAGER) F32Vec<V>::store(a.dpl + at, d);
-      if (VAR != VAR_STANDARD && m == 0) F32Vec<V>::store(a.dpa + i, mean);
-    }
-  }
-  if (blockIdx.x == gridDim.x - 1) { // ragged tail, one index per thread
-    const long long t = nvec * V + threadIdx.x;
-    if (t < a.P) outer_column_rt<VAR, TK, BOOT, 1, Q>(a, t);
+    if (t < a.P) outer_column_rt<VAR, TK, false, 1, Q>(a, t);
   }
 }
 

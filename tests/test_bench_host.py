@@ -34,3 +34,37 @@ def test_reference_arm_prints_one_json_line():
     assert d["impl"] == "reference" and d["metric"] == bench.METRIC and d["unit"] == bench.UNIT
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
     assert d["value"] > 0 and d["gpu_launches"] == 0
+
+
+def test_both_arms_describe_the_workload_identically():
+    """The GPU arm and the CPU reference arm must print the same `config` for the same command
+    line, so that a reader (or a driver) comparing the two lines sees one workload."""
+    import argparse
+    from paper_2502_12996_b200 import inputs
+    args = argparse.Namespace(workload=bench.DEFAULT_WORKLOAD, variant="eager", outer_only=False, strong=False, kernel=0,
+                              comm="f32")
+    w = inputs.WORKLOADS[bench.DEFAULT_WORKLOAD]
+    cfg = bench.config_dict(args, w, w.P)
+    assert cfg["workload"] == "cfg4a" and cfg["M"] == 2 and cfg["P_per_gpu"] == 2_400_000_000
+    out = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "1",
+                          "--workload", "cfg0"], capture_output=True, text=True, timeout=300, check=True).stdout
+    d = json.loads(out.strip().splitlines()[-1])
+    args.workload = "cfg0"
+    assert d["config"] == bench.config_dict(args, inputs.WORKLOADS["cfg0"], inputs.WORKLOADS["cfg0"].P)
+    assert "cold-L2" in d["config"]["l2"]                         # 37.7 MB of state: smaller than L2
+    assert "state >> 126 MB L2" in cfg["l2"]
+
+
+def test_traffic_table_parses():
+    table = bench.load_traffic()
+    assert ("outer", "eager", 4, 0) in table
+    for (kernel, variant, M, kind), (bpp, source) in table.items():
+        assert kernel in ("outer", "adamw") and 1 <= M <= 64 and kind in (0, 1, 2) and bpp > 0
+        assert (ROOT / "profiles" / source).exists(), source
+
+
+def test_oracle_sample_is_bounded():
+    from paper_2502_12996_b200 import inputs
+    for w in inputs.WORKLOADS.values():
+        n = bench.oracle_sample_size(w, w.P)
+        assert n <= w.P and n * w.M <= 140_000_000

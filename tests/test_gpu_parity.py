@@ -623,7 +623,7 @@ def test_bench_two_ranks_dry_run(tmp_path):
         port = sock.getsockname()[1]
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
            "127.0.0.1", "--master-port", str(port), str(root / "bench.py"), "--gpus", "2", "--steps", "3", "--warmup", "3",
-           "--P", "2000000", "--no-cpu-baseline", "--no-siblings"]
+           "--workload", "cfg1", "--P", "2000000", "--no-cpu-baseline"]
     out = subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env, cwd=str(root))
     assert out.returncode == 0, out.stderr[-2000:]
     lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
@@ -648,7 +648,8 @@ def test_bench_line_has_every_contract_key():
     for k in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
               "vs_baseline", "dtype", "data", "config", "roofline", "cpu_baseline", "e2e", "gpu_launches", "clocks"):
         assert k in d, k
-    assert d["config"]["workload"] == "cfg1" and d["vs_baseline"] is None and d["data"] == "synthetic"
+    assert d["config"]["workload"] == "cfg4a" and d["config"]["M"] == 2            # the default: largest outer-only shape
+    assert d["vs_baseline"] is None and d["data"] == "synthetic" and d["shapes"] is None   # --P: one shape only
     assert d["n_gpus"] == 1 and d["steps"] == 3 and d["gpu_launches"] == 3 and d["higher_is_better"] is True
     for k in ("bound", "achieved", "peak", "unit", "frac", "traffic"):
         assert k in d["roofline"], k
@@ -658,7 +659,8 @@ def test_bench_line_has_every_contract_key():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
     for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step"):
         assert k in d["e2e"], k
-    assert d["e2e"]["h2d_bytes_per_step"] == 3000000 * (4 * 16 + 4) and d["e2e"]["value"] < d["value"]
+    assert d["e2e"]["h2d_bytes_per_step"] == 3000000 * (4 * 8 + 4) and d["e2e"]["value"] < d["value"]
+    assert d["e2e"]["workload"] == "cfg4a"
     for k in ("sm_mhz", "sm_max_mhz", "reasons"):
         assert k in d["clocks"], k
 
