@@ -45,6 +45,8 @@ struct diloco_state {
   int64_t outer_step;
   int32_t have_prev;
   std::vector<Fragment> frags;
+  const void *checked[8]; // per-call buffers already seen to be memory of this device (H calls per phase
+  int checked_next;       // pass the same gradient / send / receive buffers again and again)
   uint64_t wait_limit_ns;  // bound of every device-side wait of the bulk form
   uint32_t test_extra_tx;  // bytes its barriers over-expect: 0 except in the give-up test
   std::vector<cudaEvent_t> events; // host-path chunk events, created on first use
@@ -105,6 +107,19 @@ int check_device_pointer(const void *p, int device) {
   }
   if (at.type == cudaMemoryTypeManaged) return DILOCO_OK;
   if (at.type != cudaMemoryTypeDevice || at.device != device) return DILOCO_ERR_INVALID_ARG;
+  return DILOCO_OK;
+}
+
+// Per-call buffers (gradients, send / receive buffers) are checked once per address and state:
+// a training loop passes the same few buffers at every step, and the attribute query is a
+// driver call on the launch path.
+int check_call_pointer(diloco_state *st, const void *p) {
+  for (const void *q : st->checked)
+    if (q == p) return DILOCO_OK;
+  const int rc = check_device_pointer(p, st->device);
+  if (rc != DILOCO_OK) return rc;
+  st->checked[st->checked_next] = p;
+  st->checked_next = (st->checked_next + 1) % 8;
   return DILOCO_OK;
 }
 
@@ -457,6 +472,8 @@ int diloco_state_init(const diloco_config_t *config, const diloco_buffers_t *buf
   st->inner_step = 0;
   st->outer_step = 0;
   st->have_prev = config->have_prev;
+  for (const void *&q : st->checked) q = nullptr;
+  st->checked_next = 0;
   st->wait_limit_ns = kDefaultWaitLimitNs;
   st->test_extra_tx = 0;
   st->last_d2h = nullptr;
@@ -482,7 +499,7 @@ int diloco_inner_adamw(diloco_state_t *st, const void *grads, int64_t grad_strid
   }
   const size_t gelt = st->cfg.grad_kind == DILOCO_GRAD_F32 ? 4 : 2;
   if (!aligned16(grads) || (grad_stride * (int64_t)gelt) % 128 != 0) return DILOCO_ERR_MISALIGNED;
-  if (check_device_pointer(grads, st->device) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
+  if (check_call_pointer(st, grads) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
   const int64_t k = st->inner_step + 1;
   AdamArgs a;
   a.theta = st->buf.theta;
@@ -575,7 +592,7 @@ int diloco_worker_outer_send(diloco_state_t *st, float *delta_send, void *stream
   if (!aligned16(delta_send)) return DILOCO_ERR_MISALIGNED;
   int rc = check_device(st);
   if (rc != DILOCO_OK) return rc;
-  if (check_device_pointer(delta_send, st->device) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
+  if (check_call_pointer(st, delta_send) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
   WorkerArgs a = worker_args(st, 1, nullptr, delta_send);
   return launch_worker<WMODE_SEND_ONLY, VAR_STANDARD>(st->cfg.theta_kind, a, static_cast<cudaStream_t>(stream));
 }
@@ -593,8 +610,8 @@ int diloco_worker_outer_apply(diloco_state_t *st, int32_t variant, int32_t world
   if ((delta_send && !aligned16(delta_send)) || (delta_sum_recv && !aligned16(delta_sum_recv))) return DILOCO_ERR_MISALIGNED;
   int rc = check_device(st);
   if (rc != DILOCO_OK) return rc;
-  if (delta_send && check_device_pointer(delta_send, st->device) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
-  if (!first && check_device_pointer(delta_sum_recv, st->device) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
+  if (delta_send && check_call_pointer(st, delta_send) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
+  if (!first && check_call_pointer(st, delta_sum_recv) != DILOCO_OK) return DILOCO_ERR_INVALID_ARG;
   WorkerArgs a = worker_args(st, world_replicas, delta_sum_recv, delta_send);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int tk = st->cfg.theta_kind;
@@ -619,7 +636,7 @@ int diloco_worker_quantized_send(diloco_state_t *st, int32_t exp_bits, int32_t m
   if ((reinterpret_cast<uintptr_t>(payload_send) & 3u) || (reinterpret_cast<uintptr_t>(amax_send) & 3u)) return DILOCO_ERR_MISALIGNED;
   int rc = check_device(st);
   if (rc != DILOCO_OK) return rc;
-  if (check_device_pointer(payload_send, st->device) != DILOCO_OK || check_device_pointer(amax_send, st->device) != DILOCO_OK)
+  if (check_call_pointer(st, payload_send) != DILOCO_OK || check_call_pointer(st, amax_send) != DILOCO_OK)
     return DILOCO_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   rc = launch_worker_amax(st, amax_send, s);
@@ -651,11 +668,11 @@ int diloco_worker_quantized_apply(diloco_state_t *st, int32_t variant, int32_t w
   if (sends && ((reinterpret_cast<uintptr_t>(payload_send) & 3u) || (reinterpret_cast<uintptr_t>(amax_send) & 3u))) return DILOCO_ERR_MISALIGNED;
   int rc = check_device(st);
   if (rc != DILOCO_OK) return rc;
-  if (!first && (check_device_pointer(payloads_recv, st->device) != DILOCO_OK ||
-                 check_device_pointer(amaxes_recv, st->device) != DILOCO_OK))
+  if (!first && (check_call_pointer(st, payloads_recv) != DILOCO_OK ||
+                 check_call_pointer(st, amaxes_recv) != DILOCO_OK))
     return DILOCO_ERR_INVALID_ARG;
-  if (sends && (check_device_pointer(payload_send, st->device) != DILOCO_OK ||
-                check_device_pointer(amax_send, st->device) != DILOCO_OK))
+  if (sends && (check_call_pointer(st, payload_send) != DILOCO_OK ||
+                check_call_pointer(st, amax_send) != DILOCO_OK))
     return DILOCO_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (sends) {

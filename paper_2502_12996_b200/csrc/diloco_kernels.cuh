@@ -117,6 +117,11 @@ __device__ __forceinline__ float bf16_bits_to_f32(unsigned short h) { return __u
 __device__ __forceinline__ unsigned short f32_to_bf16_bits(float f) {
   return __bfloat16_as_ushort(__float2bfloat16_rn(f)); // round-to-nearest-even
 }
+// two values in one conversion instruction: lo in bits 0-15, hi in bits 16-31 (same rounding)
+__device__ __forceinline__ unsigned f32x2_to_bf16x2_bits(float lo, float hi) {
+  const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const unsigned *>(&t);
+}
 
 template <int V> struct BF16Vec;
 template <> struct BF16Vec<8> {
@@ -132,7 +137,7 @@ template <> struct BF16Vec<8> {
   static __device__ __forceinline__ void store(unsigned short *p, const float (&r)[8]) {
     unsigned w[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) w[k] = (unsigned)f32_to_bf16_bits(r[2 * k]) | ((unsigned)f32_to_bf16_bits(r[2 * k + 1]) << 16);
+    for (int k = 0; k < 4; ++k) w[k] = f32x2_to_bf16x2_bits(r[2 * k], r[2 * k + 1]);
     DILOCO_STG(reinterpret_cast<uint4 *>(p), make_uint4(w[0], w[1], w[2], w[3]));
   }
 };
@@ -144,8 +149,8 @@ template <> struct BF16Vec<4> {
   }
   static __device__ __forceinline__ void store(unsigned short *p, const float (&r)[4]) {
     uint2 t;
-    t.x = (unsigned)f32_to_bf16_bits(r[0]) | ((unsigned)f32_to_bf16_bits(r[1]) << 16);
-    t.y = (unsigned)f32_to_bf16_bits(r[2]) | ((unsigned)f32_to_bf16_bits(r[3]) << 16);
+    t.x = f32x2_to_bf16x2_bits(r[0], r[1]);
+    t.y = f32x2_to_bf16x2_bits(r[2], r[3]);
     DILOCO_STG(reinterpret_cast<uint2 *>(p), t);
   }
 };
@@ -155,7 +160,7 @@ template <> struct BF16Vec<2> {
     r[0] = bf16_bits_to_f32(t & 0xffffu); r[1] = bf16_bits_to_f32(t >> 16);
   }
   static __device__ __forceinline__ void store(unsigned short *p, const float (&r)[2]) {
-    DILOCO_STG(reinterpret_cast<unsigned *>(p), (unsigned)f32_to_bf16_bits(r[0]) | ((unsigned)f32_to_bf16_bits(r[1]) << 16));
+    DILOCO_STG(reinterpret_cast<unsigned *>(p), f32x2_to_bf16x2_bits(r[0], r[1]));
   }
 };
 template <> struct BF16Vec<1> {
