@@ -87,7 +87,13 @@ enum {
   /* force one of the warp-split forms (replica axis over the warps of a block) whatever M is,
      for measurements; AUTO picks among them and the per-M shapes by M */
   DILOCO_IMPL_SPLIT_R2 = 3, /* two replicas per warp, 128-bit accesses (M <= 32, else as AUTO) */
-  DILOCO_IMPL_SPLIT_R4 = 4  /* four replicas per warp, 64-bit accesses                          */
+  DILOCO_IMPL_SPLIT_R4 = 4, /* four replicas per warp, 64-bit accesses                          */
+  /* tiles [M replicas x T indices] of every buffer moved by 2-D TMA box copies (tensor maps over
+     this GPU's memory, no multicast), updated in shared memory; fp32 theta only, needs
+     device_status; other states and first steps take the direct form */
+  DILOCO_IMPL_TENSOR_T256 = 5,
+  DILOCO_IMPL_TENSOR_T128 = 6,
+  DILOCO_IMPL_TENSOR_T64 = 7
 };
 
 typedef struct {

@@ -17,6 +17,7 @@ OK, ERR_INVALID_ARG, ERR_MISALIGNED, ERR_BAD_STATE, ERR_CUDA, ERR_DEVICE_TIMEOUT
 THETA_F32, THETA_BF16, THETA_MASTER_BF16 = 0, 1, 2
 GRAD_F32, GRAD_BF16 = 0, 1
 IMPL_AUTO, IMPL_DIRECT, IMPL_BULK, IMPL_SPLIT_R2, IMPL_SPLIT_R4 = 0, 1, 2, 3, 4
+IMPL_TENSOR_T256, IMPL_TENSOR_T128, IMPL_TENSOR_T64 = 5, 6, 7
 STANDARD, DELAYED, EAGER = 0, 1, 2
 COMM_F32, COMM_BF16, COMM_EXMY = 0, 1, 2
 MAX_M = 64

@@ -17,6 +17,7 @@
 #include "diloco_bulk.cuh"
 #include "diloco_kernels.cuh"
 #include "diloco_outer_launch.cuh"
+#include "diloco_tensor.cuh"
 #include "diloco_worker.cuh"
 
 using namespace diloco;
@@ -82,7 +83,7 @@ int validate_config(const diloco_config_t *c) {
   if (c->M > DILOCO_MAX_M) return DILOCO_ERR_UNSUPPORTED;
   if (c->theta_kind < DILOCO_THETA_F32 || c->theta_kind > DILOCO_THETA_MASTER_BF16) return DILOCO_ERR_INVALID_ARG;
   if (c->grad_kind < DILOCO_GRAD_F32 || c->grad_kind > DILOCO_GRAD_BF16) return DILOCO_ERR_INVALID_ARG;
-  if (c->impl < DILOCO_IMPL_AUTO || c->impl > DILOCO_IMPL_SPLIT_R4) return DILOCO_ERR_INVALID_ARG;
+  if (c->impl < DILOCO_IMPL_AUTO || c->impl > DILOCO_IMPL_TENSOR_T64) return DILOCO_ERR_INVALID_ARG;
   if (!(c->outer_momentum >= 0.f && c->outer_momentum < 1.f)) return DILOCO_ERR_INVALID_ARG;
   if (!std::isfinite(c->outer_lr)) return DILOCO_ERR_INVALID_ARG;
   if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f)) return DILOCO_ERR_INVALID_ARG;
@@ -291,8 +292,95 @@ int launch_bulk_m(const diloco_state *st, int var, int tk, const OuterArgs &a, c
   });
 }
 
+// ---- tensor (2-D TMA) form ---------------------------------------------------------------------
+// cuTensorMapEncodeTiled is a driver entry point; it is looked up through the runtime so that the
+// library needs no link-time dependency on the driver library.
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static std::once_flag once;
+  static EncodeTiledFn fn = nullptr;
+  std::call_once(once, [] {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      cudaGetLastError();
+  });
+  return fn;
+}
+
+// fp32 tensor [rows, cols] with row pitch `pitch` elements, boxes of [rows, T]
+int encode_rows(CUtensorMap *map, float *base, int64_t cols, int rows, int64_t pitch, int T) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return DILOCO_ERR_UNSUPPORTED;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)pitch * sizeof(float)};
+  const cuuint32_t box[2] = {(cuuint32_t)T, (cuuint32_t)rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? DILOCO_OK : DILOCO_ERR_CUDA;
+}
+
+template <int VAR, int T>
+int launch_tensor_t(const diloco_state *st, const OuterArgs &whole, cudaStream_t s) {
+  constexpr int NT = 256;
+  auto k = outer_step_tensor_kernel<VAR, T, NT>;
+  const int M = st->cfg.M;
+  const size_t stage = (size_t)tensor_rows_per_stage<VAR>(M) * T * sizeof(float);
+  const size_t budget = 227 * 1024 - 1024; // dynamic shared memory of one CTA, static part left out
+  int stages = (int)(budget / stage);
+  if (stages > kTensorMaxStages) stages = kTensorMaxStages;
+  if (stages < 3) return DILOCO_ERR_UNSUPPORTED;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(stage * stages));
+  if (e != cudaSuccess) return cuda_fail(e);
+  // TMA coordinates are 32-bit: segments of at most 2^30 columns, each with tensor maps of its own
+  const long long seg = 1ll << 30;
+  for (long long off = 0; off < whole.P; off += seg) {
+    OuterArgs a = whole;
+    a.P = whole.P - off < seg ? whole.P - off : seg;
+    TensorMaps maps;
+    int rc = encode_rows(&maps.theta, reinterpret_cast<float *>(whole.theta) + off, a.P, M, a.stride, T);
+    if (rc == DILOCO_OK) rc = encode_rows(&maps.start, whole.start + off, a.P, M, a.stride, T);
+    if (rc == DILOCO_OK) rc = encode_rows(&maps.mom, whole.mom + off, a.P, M, a.stride, T);
+    if (rc == DILOCO_OK && VAR == VAR_EAGER) rc = encode_rows(&maps.dpl, whole.dpl + off, a.P, M, a.stride, T);
+    if (rc == DILOCO_OK && VAR != VAR_STANDARD) rc = encode_rows(&maps.dpa, whole.dpa + off, a.P, 1, a.stride, T);
+    if (rc != DILOCO_OK) return rc;
+    long long grid = st->sm_count;
+    const long long ntiles = (a.P + T - 1) / T;
+    if (grid > ntiles) grid = ntiles;
+    k<<<(unsigned)grid, NT, stage * stages, s>>>(maps, a, st->buf.device_status, stages, (unsigned long long)st->wait_limit_ns,
+                                                 st->test_extra_tx);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_launches.fetch_add(1);
+  }
+  return DILOCO_OK;
+}
+
+template <int T>
+int launch_tensor(const diloco_state *st, int var, const OuterArgs &a, cudaStream_t s) {
+  if (var == VAR_STANDARD) return launch_tensor_t<VAR_STANDARD, T>(st, a, s);
+  if (var == VAR_DELAYED) return launch_tensor_t<VAR_DELAYED, T>(st, a, s);
+  return launch_tensor_t<VAR_EAGER, T>(st, a, s);
+}
+
 int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t len, cudaStream_t s, int ring = -1) {
   OuterArgs a = outer_args(st, offset, len, ring);
+  // The tensor form: fp32 theta, needs the status word for its bounded waits; falls back to the
+  // direct form where a stage ring of three tiles does not fit shared memory.
+  if (st->cfg.impl >= DILOCO_IMPL_TENSOR_T256 && st->cfg.impl <= DILOCO_IMPL_TENSOR_T64 && !boot &&
+      st->buf.device_status && st->cfg.theta_kind == DILOCO_THETA_F32) {
+    int rc = DILOCO_ERR_UNSUPPORTED;
+    if (st->cfg.impl == DILOCO_IMPL_TENSOR_T256) rc = launch_tensor<256>(st, var, a, s);
+    else if (st->cfg.impl == DILOCO_IMPL_TENSOR_T128) rc = launch_tensor<128>(st, var, a, s);
+    else rc = launch_tensor<64>(st, var, a, s);
+    if (rc != DILOCO_ERR_UNSUPPORTED) return rc;
+  }
   // The bulk form exists for M = 2 and M = 4 only, needs the status word for its bounded
   // waits and at least one full tile; everything else (and AUTO) takes the direct form,
   // which measured faster at every M.
@@ -890,7 +978,7 @@ int diloco_set_outer_hparams(diloco_state_t *st, float outer_lr, float outer_mom
 }
 
 int diloco_set_impl(diloco_state_t *st, int32_t impl) {
-  if (!st || impl < DILOCO_IMPL_AUTO || impl > DILOCO_IMPL_SPLIT_R4) return DILOCO_ERR_INVALID_ARG;
+  if (!st || impl < DILOCO_IMPL_AUTO || impl > DILOCO_IMPL_TENSOR_T64) return DILOCO_ERR_INVALID_ARG;
   st->cfg.impl = impl;
   return DILOCO_OK;
 }

@@ -100,8 +100,41 @@ def test_bulk_staged_implementation(oracle, variant, theta_kind, M, P):
     run_outer_steps(oracle, variant, M, P, theta_kind, steps=3, seed=650 + M, impl=binding.IMPL_BULK)
 
 
-@pytest.mark.parametrize("M,P", [(2, 8 * 1024 + 5), (4, 40 * 512)])
-def test_bounded_device_wait_runs_out_and_is_reported(oracle, M, P):
+@pytest.mark.parametrize("impl", [binding.IMPL_TENSOR_T256, binding.IMPL_TENSOR_T128, binding.IMPL_TENSOR_T64])
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("M,P", [(1, 70_001), (2, 300_003), (4, 200_005), (5, 9_999), (8, 60_001), (16, 50_003), (4, 255),
+                                 (3, 1)])
+def test_tensor_map_implementation(oracle, impl, variant, M, P):
+    """The 2-D TMA form (one box copy per buffer and tile, all M replicas at once; columns
+    beyond P zero-filled on load and clipped on store by the hardware) must give the oracle's
+    bits, ragged sizes and sizes below one tile included."""
+    run_outer_steps(oracle, variant, M, P, 0, steps=3, seed=670 + M, impl=impl)
+
+
+def test_tensor_map_implementation_large_m_and_fragments(oracle):
+    """M = 32 and 64 (narrow tiles only: three stages of wider ones do not fit shared memory and
+    the call falls back to the direct form), and a fragment whose base is not at column 0."""
+    run_outer_steps(oracle, 2, 32, 20_001, 0, steps=2, seed=680, impl=binding.IMPL_TENSOR_T128)
+    run_outer_steps(oracle, 2, 64, 9_001, 0, steps=2, seed=681, impl=binding.IMPL_TENSOR_T64)
+    run_outer_steps(oracle, 2, 64, 9_001, 0, steps=2, seed=682, impl=binding.IMPL_TENSOR_T256)   # falls back
+    M, P = 4, 100_003
+    a, _ = make(M, P, 683, 0)
+    b = {k: (v.clone() if torch.is_tensor(v) else v) for k, v in a.items()}
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sa = binding.State.from_dict(a)
+    sb = binding.State.from_dict(b, impl=binding.IMPL_TENSOR_T128, device_status=status)
+    sa.outer_eager()
+    for lo, hi in ((64 * 700, P), (0, 64 * 700)):
+        sb.outer_fragment(binding.EAGER, False, lo, hi - lo)
+    sb.check_device_status()
+    torch.cuda.synchronize()
+    for k in ("theta", "start", "delta_prev_local", "delta_prev_avg", "outer_mom"):
+        assert torch.equal(a[k].view(torch.int32), b[k].view(torch.int32)), k
+
+
+@pytest.mark.parametrize("M,P,impl", [(2, 8 * 1024 + 5, binding.IMPL_BULK), (4, 40 * 512, binding.IMPL_BULK),
+                                      (4, 20_001, binding.IMPL_TENSOR_T128), (16, 3_001, binding.IMPL_TENSOR_T64)])
+def test_bounded_device_wait_runs_out_and_is_reported(oracle, M, P, impl):
     """The staged form's only device-side waits are on mbarriers that the copy engine completes.
     Here every barrier is told to expect 16 bytes more than its copies deliver: all copies land,
     no wait can complete, every wait gives up after the 2 ms limit, the CTAs drain and return.
@@ -111,7 +144,7 @@ def test_bounded_device_wait_runs_out_and_is_reported(oracle, M, P):
     st, checks = make(M, P, 660 + M, 0)
     h = host_copy(st)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    state = binding.State.from_dict(st, impl=binding.IMPL_BULK, device_status=status)
+    state = binding.State.from_dict(st, impl=impl, device_status=status)
     state.set_wait_limit(2_000_000, 16)
     torch.cuda.synchronize()
     t0 = time.perf_counter()
