@@ -44,6 +44,8 @@ FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 << 20
 DEFAULT_WORKLOAD = "cfg4a"
 THETA_NAMES = ["f32", "bf16", "f32 master + bf16 copy"]
+KERNEL_IMPLS = ["auto", "direct", "bulk (1-D TMA rows)", "split R2", "split R4", "tensor (2-D TMA) T256", "tensor T128",
+                "tensor T64"]
 VARIANTS = {"standard": 0, "delayed": 1, "eager": 2}
 # measured DRAM traffic per parameter index, one row per profiled kernel form
 TRAFFIC_TABLE = ROOT / "profiles" / "ncu_dram_bytes_per_index.txt"
@@ -203,7 +205,7 @@ def config_dict(args, w, P_per_gpu: int) -> dict:
             "outer_lr": w.outer_lr, "outer_momentum": w.outer_momentum, "l2": l2,
             "sharding": "one full shape per rank (weak scaling), all M replicas of an index on one rank, no collective"
             if not args.strong else "parameter axis split across ranks, all M replicas of an index on one rank, no collective",
-            "kernel_impl": ["auto", "direct", "bulk"][args.kernel], "outer_gradient_wire_format": args.comm}
+            "kernel_impl": KERNEL_IMPLS[args.kernel], "outer_gradient_wire_format": args.comm}
 
 
 # ------------------------------------------------------------------------------------ CPU arm
@@ -309,7 +311,7 @@ class Shape:
         self.comm = COMM[comm]
         self.kernel = args.kernel
         self.seed = w.seed + 1000 * rank
-        self.st = self.state = self.grads = self.scratch = None
+        self.st = self.state = self.grads = self.scratch = self.status = None
 
     def need_bytes(self):
         w, M, P = self.w, self.w.M, self.P
@@ -332,6 +334,9 @@ class Shape:
         if self.comm[0]:
             self.scratch = torch.zeros(64, dtype=torch.int32, device=self.dev)
             kw["comm_scratch"] = self.scratch
+        if self.kernel in (2, 5, 6, 7):                     # the staged forms report a timed-out wait here
+            self.status = torch.zeros(1, dtype=torch.int32, device=self.dev)
+            kw["device_status"] = self.status
         self.state = binding.State.from_dict(st, **kw)
         if self.phase:
             if w.segments:
@@ -403,6 +408,7 @@ class Shape:
         launches = binding.launch_count() - n0
         if barrier:
             barrier()
+        self.state.check_device_status()                    # raises if a staged form gave up a wait
         return rows, launches, sampler.window(t0, t1, t_warm)
 
     def record(self, rows, clocks, peak, traffic):
@@ -790,7 +796,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--variant", default="eager", choices=list(VARIANTS))
     ap.add_argument("--P", type=int, default=0, help="override the workload's parameter count (per GPU)")
-    ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 direct, 2 bulk")
+    ap.add_argument("--kernel", type=int, default=0, choices=range(len(KERNEL_IMPLS)),
+                    help="kernel form, DILOCO_IMPL_*: " + ", ".join(f"{i} {n}" for i, n in enumerate(KERNEL_IMPLS)))
     ap.add_argument("--comm", default="f32", choices=list(COMM),
                     help="wire format of the outer gradients (quantised communication)")
     ap.add_argument("--chunk", type=int, default=64 * 16384, help="elements per chunk of the host-buffer path")

@@ -343,16 +343,30 @@ int launch_tensor_t(const diloco_state *st, const OuterArgs &whole, cudaStream_t
   for (long long off = 0; off < whole.P; off += seg) {
     OuterArgs a = whole;
     a.P = whole.P - off < seg ? whole.P - off : seg;
+    a.theta = reinterpret_cast<float *>(whole.theta) + off;
+    a.start = whole.start + off;
+    a.mom = whole.mom + off;
+    a.dpl = whole.dpl ? whole.dpl + off : nullptr;
+    a.dpa = whole.dpa ? whole.dpa + off : nullptr;
+    // the tensors end at a multiple of 4 columns (16 bytes: the unit in which stores are clipped);
+    // the kernel's last CTA does the remaining P % 4 indices itself
+    const long long cols = a.P & ~3ll;
     TensorMaps maps;
-    int rc = encode_rows(&maps.theta, reinterpret_cast<float *>(whole.theta) + off, a.P, M, a.stride, T);
-    if (rc == DILOCO_OK) rc = encode_rows(&maps.start, whole.start + off, a.P, M, a.stride, T);
-    if (rc == DILOCO_OK) rc = encode_rows(&maps.mom, whole.mom + off, a.P, M, a.stride, T);
-    if (rc == DILOCO_OK && VAR == VAR_EAGER) rc = encode_rows(&maps.dpl, whole.dpl + off, a.P, M, a.stride, T);
-    if (rc == DILOCO_OK && VAR != VAR_STANDARD) rc = encode_rows(&maps.dpa, whole.dpa + off, a.P, 1, a.stride, T);
+    int rc = DILOCO_OK;
+    if (cols > 0) {
+      rc = encode_rows(&maps.theta, reinterpret_cast<float *>(a.theta), cols, M, a.stride, T);
+      if (rc == DILOCO_OK) rc = encode_rows(&maps.start, a.start, cols, M, a.stride, T);
+      if (rc == DILOCO_OK) rc = encode_rows(&maps.mom, a.mom, cols, M, a.stride, T);
+      if (rc == DILOCO_OK && VAR == VAR_EAGER) rc = encode_rows(&maps.dpl, a.dpl, cols, M, a.stride, T);
+      if (rc == DILOCO_OK && VAR != VAR_STANDARD) rc = encode_rows(&maps.dpa, a.dpa, cols, 1, a.stride, T);
+    } else {
+      std::memset(&maps, 0, sizeof(maps)); // fewer than 4 indices: no tile, the maps are never used
+    }
     if (rc != DILOCO_OK) return rc;
     long long grid = st->sm_count;
-    const long long ntiles = (a.P + T - 1) / T;
+    const long long ntiles = (cols + T - 1) / T;
     if (grid > ntiles) grid = ntiles;
+    if (grid < 1) grid = 1;
     k<<<(unsigned)grid, NT, stage * stages, s>>>(maps, a, st->buf.device_status, stages, (unsigned long long)st->wait_limit_ns,
                                                  st->test_extra_tx);
     e = cudaGetLastError();
@@ -376,9 +390,11 @@ int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t l
   if (st->cfg.impl >= DILOCO_IMPL_TENSOR_T256 && st->cfg.impl <= DILOCO_IMPL_TENSOR_T64 && !boot &&
       st->buf.device_status && st->cfg.theta_kind == DILOCO_THETA_F32) {
     int rc = DILOCO_ERR_UNSUPPORTED;
-    if (st->cfg.impl == DILOCO_IMPL_TENSOR_T256) rc = launch_tensor<256>(st, var, a, s);
-    else if (st->cfg.impl == DILOCO_IMPL_TENSOR_T128) rc = launch_tensor<128>(st, var, a, s);
-    else rc = launch_tensor<64>(st, var, a, s);
+    switch (st->cfg.impl) {
+      case DILOCO_IMPL_TENSOR_T256: rc = launch_tensor<256>(st, var, a, s); break;
+      case DILOCO_IMPL_TENSOR_T128: rc = launch_tensor<128>(st, var, a, s); break;
+      default: rc = launch_tensor<64>(st, var, a, s); break;
+    }
     if (rc != DILOCO_ERR_UNSUPPORTED) return rc;
   }
   // The bulk form exists for M = 2 and M = 4 only, needs the status word for its bounded

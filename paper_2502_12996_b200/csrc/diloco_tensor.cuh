@@ -4,8 +4,11 @@
 // A tile therefore costs 5 loads and 5 stores (theta, start, outer_mom, delta_prev_local,
 // delta_prev_avg) whatever M is, where the row-by-row form of diloco_bulk.cuh needs 4 M + 1 of
 // each - the per-copy cost of the copy engine was what limited that form.  The tensor maps cover
-// this GPU's own memory only and no copy uses cluster multicast.  Columns at and beyond P are
-// zero-filled on load and clipped on store by the hardware, so there is no ragged-tail code.
+// this GPU's own memory only and no copy uses cluster multicast.  The tensors cover the columns
+// [0, P4), P4 = P rounded down to a multiple of 4: the hardware zero-fills a box's columns
+// beyond that on load and clips them on store, but it clips in units of 16 bytes, so a tensor
+// that ended inside a 16-byte unit would have its padding overwritten.  The last P % 4 indices
+// are done with plain loads and stores by the last CTA.
 //
 // Per CTA (one per SM, tiles taken round-robin), ring of S stages:
 //   thread 0:  arm full[s] with the tile's byte count, issue the box loads (complete_tx)
@@ -16,6 +19,13 @@
 //   thread 0:  issue the box stores as one bulk group; before a stage is refilled, wait until
 //              the group that drained it has finished reading shared memory
 // Same arithmetic, same order, same bits as the direct form.  fp32 theta, M at run time.
+// Measured (eager fp32, GB/s; direct form in brackets): T = 256: M = 2 2548 [6760], M = 4 4401
+// [6773], M = 8 6163-6573 [6729], M = 16 6250 [6554], M = 32 falls back.  One CTA per SM works
+// through its tiles one after the other, so below M = 8 the per-tile latency of the two passes
+// (about 1 us) is not hidden by anything, and at M = 16 only three 68 KB stages fit, i.e. one
+// tile of loads in flight.  A hybrid with TMA loads and ordinary stores from registers (half the
+// box copies, one more stage for loads) measured the same or lower (M = 8 6380, M = 16 5903) and
+// was dropped.  The form is kept as a tested alternative; AUTO never selects it.
 #pragma once
 #include <cuda.h>
 
@@ -61,7 +71,8 @@ __global__ void __launch_bounds__(NT, 1)
 
   const int M = a.M, S = stages, tid = threadIdx.x;
   const int rows = tensor_rows_per_stage<VAR>(M);
-  const long long ntiles = (a.P + T - 1) / T;
+  const long long P4 = a.P & ~3ll;                 // columns the tensor maps cover
+  const long long ntiles = (P4 + T - 1) / T;
   const long long mine = ntiles > blockIdx.x ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
   const int LOOK = S - 2; // tiles in flight ahead of the one being computed; one more stage is draining
   // stage layout, in floats
@@ -181,6 +192,11 @@ __global__ void __launch_bounds__(NT, 1)
   if (tid == 0) {
     bulk_wait_all();
     if (aborted && status) atomicExch(status, kStatusTimeout);
+  }
+  // ragged remainder (P % 4 indices): plain loads and stores, one index per thread
+  if (blockIdx.x == gridDim.x - 1 && !aborted) {
+    const long long i = P4 + tid;
+    if (i < a.P) outer_column_rt<VAR, TK_F32, false, 1>(a, i);
   }
 }
 

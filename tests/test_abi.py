@@ -67,7 +67,7 @@ def init(lib, cfg, buf):
 
 @pytest.mark.parametrize("kw", [dict(M=0), dict(M=-3), dict(P=0), dict(stride=999), dict(theta_kind=3), dict(grad_kind=2),
                                 dict(outer_momentum=1.0), dict(outer_momentum=-0.1), dict(beta1=1.0), dict(beta2=-1.0),
-                                dict(eps=-1e-8), dict(weight_decay=-1.0), dict(have_prev=2), dict(impl=9), dict(impl=-1),
+                                dict(eps=-1e-8), dict(weight_decay=-1.0), dict(have_prev=2), dict(impl=8), dict(impl=-1),
                                 dict(outer_lr=float("nan")), dict(H=-1), dict(overlap_steps=0), dict(have_prev=-1),
                                 dict(overlap_steps=2, have_prev=3)])
 def test_invalid_config(lib, kw):
