@@ -438,16 +438,35 @@ class Shape:
         return rec
 
 
-def register_host(torch, t):
-    """Page-lock a host tensor in place (exact size: the caching pinned allocator rounds every
-    request up to a power of two, which would double an 86 GB state)."""
-    rc = torch.cuda.cudart().cudaHostRegister(t.data_ptr(), t.numel() * t.element_size(), 0)
-    if int(rc) != 0:
-        raise RuntimeError(f"cudaHostRegister failed with {rc}")
+class HostBuffer:
+    """A page-locked host tensor of exactly the size asked for.  The caching pinned allocator
+    rounds every request up to a power of two, which would double an 86 GB state, so the memory
+    is an anonymous mapping that is advised to use huge pages (on this pool plain 4 KB pages cost
+    the copies 15-20 % of their PCIe rate: 35 against 43 GB/s each way) and then page-locked in
+    place with cudaHostRegister."""
 
+    def __init__(self, torch, like):
+        import mmap
+        self.torch = torch
+        nbytes = like.numel() * like.element_size()
+        huge = 2 << 20
+        self.map = mmap.mmap(-1, max(huge, (nbytes + huge - 1) // huge * huge))
+        try:
+            self.map.madvise(mmap.MADV_HUGEPAGE)
+        except (AttributeError, OSError, ValueError):
+            pass                                            # no transparent huge pages here: 4 KB pages then
+        self.tensor = torch.frombuffer(self.map, dtype=like.dtype, count=like.numel()).view(like.shape)
+        rc = torch.cuda.cudart().cudaHostRegister(self.tensor.data_ptr(), nbytes, 0)
+        if int(rc) != 0:
+            raise RuntimeError(f"cudaHostRegister failed with {rc}")
+        self.tensor.copy_(like)
 
-def unregister_host(torch, t):
-    torch.cuda.cudart().cudaHostUnregister(t.data_ptr())
+    def release(self):
+        try:
+            self.torch.cuda.cudart().cudaHostUnregister(self.tensor.data_ptr())
+        except Exception:
+            pass
+        self.tensor = None                                  # the mapping goes with the last reference to it
 
 
 def run_e2e(shape, args, world, dist, red_dev, n_steps):
@@ -457,15 +476,14 @@ def run_e2e(shape, args, world, dist, red_dev, n_steps):
     torch, binding = shape.torch, shape.binding
     st, w, P, M, variant = shape.st, shape.w, shape.P, shape.w.M, shape.variant
     keys = ("theta", "master", "start", "delta_prev_local", "delta_prev_avg", "outer_mom")
-    pinned, t_pin = {}, time.perf_counter()
+    pinned, owners, t_pin = {}, [], time.perf_counter()
     try:
         for k in keys:
             if st.get(k) is None:
                 pinned[k] = None
                 continue
-            pinned[k] = torch.empty(st[k].shape, dtype=st[k].dtype, device="cpu")
-            register_host(torch, pinned[k])
-            pinned[k].copy_(st[k])
+            owners.append(HostBuffer(torch, st[k]))
+            pinned[k] = owners[-1].tensor
         t_pin = time.perf_counter() - t_pin
         host = binding.make_buffers(**pinned)
         streams = [torch.cuda.Stream(device=shape.dev) for _ in range(3)]
@@ -500,7 +518,8 @@ def run_e2e(shape, args, world, dist, red_dev, n_steps):
                "workload": shape.name, "M": M, "P_per_gpu": P, "ms_per_step": e_ms, "steps": len(per), "chunk": args.chunk,
                "call": "diloco_outer_step_host: whole state in pinned host memory, copied in and out every step",
                "timing": "CUDA events: first copy-in stream to last copy-out stream",
-               "pcie_GBps_each_way": h2d / e_ms / 1e6, "host_register_s": t_pin}
+               "pcie_GBps_each_way": h2d / e_ms / 1e6, "host_register_s": t_pin,
+               "host_memory": "anonymous mappings advised to huge pages, page-locked with cudaHostRegister"}
         # second flavour: only theta crosses PCIe, the outer-optimiser state stays on the device
         host_t = binding.make_buffers(theta=pinned["theta"], master=pinned["master"])
         per = [host_step(host_t) for _ in range(2 + n_steps)][2:]
@@ -514,13 +533,11 @@ def run_e2e(shape, args, world, dist, red_dev, n_steps):
     except RuntimeError as ex:
         return {"value": None, "unit": UNIT, "workload": shape.name, "error": str(ex)[:200]}
     finally:
-        for t in pinned.values():
-            if t is not None:
-                try:
-                    unregister_host(torch, t)
-                except Exception:
-                    pass
+        host = host_t = None
         pinned.clear()
+        for o in owners:
+            o.release()
+        owners.clear()
         gc.collect()
 
 

@@ -347,11 +347,19 @@ int diloco_outer_fragment(diloco_state_t *state, int32_t variant, int32_t bootst
  *   advances that fragment's counters only: while its have_prev < overlap_steps a delayed /
  *   eager step records without applying, and with overlap_steps = D > 1 it consumes what this
  *   fragment recorded D of ITS OWN outer steps ago.  The state's global counters are untouched.
+ * diloco_outer_fragment_step_quantized: the same with the fragment's outer gradients rounded to
+ *   a wire format before the mean (the paper's bandwidth figures are for streaming fragments with
+ *   4-bit communication, Table 4): formats, arguments and rounding as diloco_outer_quantized; the
+ *   per-replica scale is the maximum over THIS FRAGMENT's indices, since a fragment is what one
+ *   exchange carries.  DILOCO_COMM_F32 is diloco_outer_fragment_step.  Needs comm_scratch for
+ *   DILOCO_COMM_EXMY; calls on one state must not overlap.
  * diloco_fragment_get_counters / _set_counters: per-fragment checkpoint / resume.
  * Whole-vector calls and diloco_outer_fragment (below) ignore the table.
  */
 int diloco_fragments_set(diloco_state_t *state, int32_t n, const int64_t *offsets, const int64_t *lens);
 int diloco_outer_fragment_step(diloco_state_t *state, int32_t variant, int32_t fragment_id, void *cuda_stream);
+int diloco_outer_fragment_step_quantized(diloco_state_t *state, int32_t variant, int32_t fragment_id, int32_t comm_format,
+                                         int32_t exp_bits, int32_t man_bits, void *cuda_stream);
 int diloco_fragment_get_counters(const diloco_state_t *state, int32_t fragment_id, int64_t *outer_step, int32_t *have_prev);
 int diloco_fragment_set_counters(diloco_state_t *state, int32_t fragment_id, int64_t outer_step, int32_t have_prev);
 

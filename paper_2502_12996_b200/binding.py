@@ -82,6 +82,7 @@ SYMBOLS = {
     "diloco_outer_fragment": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p]),
     "diloco_fragments_set": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)]),
     "diloco_outer_fragment_step": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
+    "diloco_outer_fragment_step_quantized": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]),
     "diloco_fragment_get_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)]),
     "diloco_fragment_set_counters": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int32]),
     "diloco_outer_step_host": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(Buffers), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int64]),
@@ -277,6 +278,11 @@ class State:
     def outer_fragment_step(self, variant, fragment_id, stream=None) -> None:
         _check(load_library().diloco_outer_fragment_step(self._handle, variant, fragment_id, _stream_ptr(stream)),
                "diloco_outer_fragment_step")
+
+    def outer_fragment_step_quantized(self, variant, fragment_id, comm_format, exp_bits=0, man_bits=0, stream=None) -> None:
+        _check(load_library().diloco_outer_fragment_step_quantized(self._handle, variant, fragment_id, comm_format, exp_bits,
+                                                                   man_bits, _stream_ptr(stream)),
+               "diloco_outer_fragment_step_quantized")
 
     def fragment_get_counters(self, fragment_id):
         a, b = ctypes.c_int64(), ctypes.c_int32()

@@ -241,8 +241,8 @@ int launch_amax_t(const diloco_state *st, const OuterArgs &a, unsigned *amax, cu
 // One quantised outer step on indices [0, P): (EXMY only) zero the per-replica maxima and
 // reduce max |Delta_m| into `scratch`, then the fused step with the wire rounding in line 8.
 int launch_outer_quantized(diloco_state *st, int var, bool boot, int comm, int X, int Y, unsigned *scratch,
-                           cudaStream_t s) {
-  OuterArgs a = outer_args(st, 0, st->cfg.P);
+                           cudaStream_t s, int64_t offset = 0, int64_t len = -1, int ring = -1) {
+  OuterArgs a = outer_args(st, offset, len < 0 ? st->cfg.P : len, ring);
   a.comm = comm;
   if (comm == COMM_EXMY) {
     a.bias = (1 << (X - 1)) - 1;
@@ -840,6 +840,29 @@ int diloco_outer_fragment_step(diloco_state_t *st, int32_t variant, int32_t frag
   const bool boot = variant != VAR_STANDARD && f.have_prev < st->cfg.overlap_steps;
   const int ring = (int)(f.outer_step % st->cfg.overlap_steps);
   rc = launch_outer(st, variant, boot, f.offset, f.len, static_cast<cudaStream_t>(stream), ring);
+  if (rc != DILOCO_OK) return rc;
+  if (boot) f.have_prev += 1;
+  f.outer_step += 1;
+  return DILOCO_OK;
+}
+
+int diloco_outer_fragment_step_quantized(diloco_state_t *st, int32_t variant, int32_t fragment_id, int32_t comm_format,
+                                         int32_t exp_bits, int32_t man_bits, void *stream) {
+  if (!st) return DILOCO_ERR_INVALID_ARG;
+  if (comm_format == DILOCO_COMM_F32) return diloco_outer_fragment_step(st, variant, fragment_id, stream);
+  int rc = check_variant(st, variant);
+  if (rc != DILOCO_OK) return rc;
+  if (fragment_id < 0 || (size_t)fragment_id >= st->frags.size()) return DILOCO_ERR_INVALID_ARG;
+  if (comm_format != DILOCO_COMM_BF16 && comm_format != DILOCO_COMM_EXMY) return DILOCO_ERR_INVALID_ARG;
+  if (comm_format == DILOCO_COMM_EXMY) {
+    if (!valid_exmy(exp_bits, man_bits)) return DILOCO_ERR_INVALID_ARG;
+    if (!st->buf.comm_scratch) return DILOCO_ERR_BAD_STATE;
+  }
+  Fragment &f = st->frags[(size_t)fragment_id];
+  const bool boot = variant != VAR_STANDARD && f.have_prev < st->cfg.overlap_steps;
+  const int ring = (int)(f.outer_step % st->cfg.overlap_steps);
+  rc = launch_outer_quantized(st, variant, boot, comm_format, exp_bits, man_bits, st->buf.comm_scratch,
+                              static_cast<cudaStream_t>(stream), f.offset, f.len, ring);
   if (rc != DILOCO_OK) return rc;
   if (boot) f.have_prev += 1;
   f.outer_step += 1;

@@ -467,6 +467,50 @@ def test_fragment_table_staggered_schedule(oracle, D, variant, theta_kind, impl)
     state.close()
 
 
+@pytest.mark.parametrize("fmt", ["e2m1", "e4m3", "bf16"])
+@pytest.mark.parametrize("D,theta_kind", [(1, 0), (2, 1)])
+def test_fragment_schedule_with_quantised_wire(oracle, fmt, D, theta_kind):
+    """Streaming fragments with a 4- or 8-bit wire, the combination behind the paper's bandwidth
+    table: each fragment's exchange is rounded with a scale of its own (the maximum over the
+    fragment's indices), on its own schedule."""
+    comm, X, Y = FORMATS[fmt]
+    M, P = 4, 30_005
+    st = inputs.make_outer_state(M, P, 1170 + D, device=DEV, theta_kind=theta_kind, overlap_steps=D)
+    stride = st["stride"]
+    h = host_copy(st)
+    h["delta_prev_local"] = h["delta_prev_local"].reshape(D, M, stride)
+    h["delta_prev_avg"] = h["delta_prev_avg"].reshape(D, stride)
+    cuts = [(0, 64 * 150), (64 * 150, 64 * 200), (64 * 350, P - 64 * 350)]
+    scratch = torch.zeros(64, dtype=torch.int32, device=DEV)
+    state = binding.State.from_dict(st, have_prev=0, overlap_steps=D, comm_scratch=scratch)
+    state.fragments_set([c[0] for c in cuts], [c[1] for c in cuts])
+    have, count = [0, 0, 0], [0, 0, 0]
+    for t in range(3 * (D + 1) + 1):
+        if t:
+            inputs.inner_phase_standin(st)
+            h["theta"], h["master"] = to_numpy(st["theta"]), to_numpy(st["master"])
+        f = t % 3
+        state.outer_fragment_step_quantized(binding.EAGER, f, comm, X, Y)
+        have[f] = oracle.outer_step_fragment(2, count[f], have[f], cuts[f][0], cuts[f][1], M=M, eta=0.7, mu=0.9,
+                                             theta=h["theta"], master=h["master"], start=h["start"],
+                                             outer_mom=h["outer_mom"], delta_prev_local=h["delta_prev_local"],
+                                             delta_prev_avg=h["delta_prev_avg"], theta_kind=theta_kind, comm=comm,
+                                             exp_bits=X, man_bits=Y)
+        count[f] += 1
+        torch.cuda.synchronize()
+        got = {key: st[key] for key in ("theta", "master", "start", "outer_mom")}
+        got["delta_prev_local"] = st["delta_prev_local"].view(D, M, stride)
+        got["delta_prev_avg"] = st["delta_prev_avg"].view(D, stride)
+        assert_state_equal(got, h, keys=tuple(got), what=f"quantised fragment schedule {fmt} D={D} t={t}")
+        assert state.fragment_get_counters(f) == (count[f], have[f])
+    no_scratch = binding.State.from_dict(st, overlap_steps=D)
+    no_scratch.fragments_set([0], [64])
+    with pytest.raises(binding.DilocoError) as e:
+        no_scratch.outer_fragment_step_quantized(binding.EAGER, 0, binding.COMM_EXMY, 4, 3)
+    assert e.value.status == binding.ERR_BAD_STATE
+    state.close()
+
+
 def test_fragment_table_argument_checks():
     st, _ = make(2, 10_000, 1160, 0, guards=False)
     state = binding.State.from_dict(st)
