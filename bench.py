@@ -418,9 +418,11 @@ class Shape:
         outer = stats([r[1] for r in rows])
         vname = [k for k, v in VARIANTS.items() if v == self.variant][0]
 
-        def kernel(name, ms, bpp, key):
+        in_l2 = state_bytes_per_param(w.M, w.theta_kind) * P <= 4 * L2_BYTES   # ncu's per-index DRAM traffic was
+
+        def kernel(name, ms, bpp, key):                                         # captured on HBM-resident sizes
             gbs = bpp * P / (ms["mean"] * 1e-3) / 1e9
-            tr = traffic.get(key)
+            tr = None if in_l2 else traffic.get(key)
             return {"kernel": name, "ms": ms, "algorithmic_bytes_per_param": bpp, "GBps": gbs, "frac": gbs / peak,
                     "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS, "GBps_best": bpp * P / (ms["min"] * 1e-3) / 1e9,
                     "ncu_dram_bytes_per_param": (tr[0] if tr else None), "ncu_profile": (tr[1] if tr else None)}
@@ -666,13 +668,18 @@ def run_ours(args):
         order = [args.workload] + [n for n in ("cfg4a", "cfg4b", "cfg4c", "cfg1", "cfg0") if n != args.workload]
         if args.P:
             order = [args.workload]
-        pick = None
-        for n in order:
+        idx = len(order)
+        for i, n in enumerate(order):
             Pn = main.P if n == args.workload else inputs.WORKLOADS[n].P
             wn = inputs.WORKLOADS[n]
             if wn.H == 0 and state_bytes_per_param(wn.M, wn.theta_kind) * Pn <= budget:
-                pick = n
+                idx = i
                 break
+        if world > 1:                                       # every rank must run the same shape: the smallest choice wins
+            t = torch.tensor([idx], device=red_dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            idx = int(t[0])
+        pick = order[idx] if idx < len(order) else None
         if pick == args.workload:
             e2e = run_e2e(main, args, world, dist, red_dev, max(3, min(args.steps, 10 if main.P < 2e8 else 3)))
         elif pick is not None:
