@@ -158,6 +158,7 @@ int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterA
       case 3: return launch_outer_shape<3, Q>(var, tk, a, s);
       case 4: return launch_outer_shape<4, Q>(var, tk, a, s);
       case 8: return launch_outer_shape<8, Q>(var, tk, a, s);
+      case 16: return launch_outer_shape<16, Q>(var, tk, a, s);
       default: break;
     }
   }
@@ -215,6 +216,8 @@ OuterArgs outer_args(const diloco_state *st, int64_t offset, int64_t len, int ri
   a.mu = st->cfg.outer_momentum;
   a.fM = (float)st->cfg.M;
   a.M = st->cfg.M;
+  a.groups = 1;
+  a.wpg = 0;
   a.amax = nullptr;
   a.fmt_max = 0.f;
   a.comm = COMM_F32;

@@ -54,17 +54,36 @@ int launch_outer_m(int var, int tk, const OuterArgs &a, cudaStream_t s) {
   });
 }
 
-// run-time M, replica axis over the warps of a block: R replicas per warp, V indices per column
+// run-time M, replica axis over the warps of a block: R replicas per warp, V indices per column,
+// two groups of columns per block where they fit 512 threads
 template <bool Q, int V, int R>
 int launch_outer_split(int var, int tk, const OuterArgs &a, cudaStream_t s) {
-  long long blocks = (a.P / V + 31) / 32;
-  if (blocks < 1) blocks = 1; // the last block also handles the P % V tail
-  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
   const int warps = (a.M + R - 1) / R;
   if (warps > 16) return DILOCO_ERR_UNSUPPORTED;
-  const size_t smem = (size_t)a.M * V * 32 * sizeof(float);
+  const int groups = (warps <= 5 || warps == 8) ? 2 : 1; // 2 x 6 or 2 x 7 warps leave a quarter of the SM's thread slots empty
+  long long blocks = ((a.P / V + 31) / 32 + groups - 1) / groups;
+  if (blocks < 1) blocks = 1; // the last block also handles the P % V tail
+  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)groups * a.M * V * 32 * sizeof(float);
+  OuterArgs b = a;
+  b.groups = groups;
+  b.wpg = warps;
   return dispatch_variant_storage(var, tk, [&](auto var_, auto tk_) {
-    outer_step_split_kernel<decltype(var_)::value, decltype(tk_)::value, Q, V, R><<<(unsigned)blocks, 32 * warps, smem, s>>>(a);
+    outer_step_split_kernel<decltype(var_)::value, decltype(tk_)::value, Q, V, R><<<(unsigned)blocks, 32 * warps * groups, smem, s>>>(b);
+    return finish_launch();
+  });
+}
+
+// M = 8 W as a chain of W warps per 16 columns
+template <bool Q, int W, int NT, int MINB>
+int launch_outer_chain(int var, int tk, const OuterArgs &a, cudaStream_t s) {
+  constexpr int GROUPS = NT / (32 * W);
+  const long long groups = (a.P / 4 + 15) / 16;
+  long long blocks = (groups + GROUPS - 1) / GROUPS;
+  if (blocks < 1) blocks = 1; // the last block also handles the P % 4 tail
+  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
+  return dispatch_variant_storage(var, tk, [&](auto var_, auto tk_) {
+    outer_step_chain_kernel<W, decltype(var_)::value, decltype(tk_)::value, NT, MINB, Q><<<(unsigned)blocks, NT, 0, s>>>(a);
     return finish_launch();
   });
 }
@@ -88,15 +107,19 @@ int launch_outer_first_steps(int var, int tk, const OuterArgs &a, cudaStream_t s
 // every warp-level access covers at least 128 contiguous bytes of a row (64-byte runs halved
 // the bandwidth).
 //   M <= 3          one thread per column, 128-bit accesses
+// and a third found later: a block should touch at least 1 KB of every row it touches (512
+// bytes per row and block cost 3 %: the DRAM pages it opens are used less fully).
 //   M = 4, 8        replica axis split over 2 lanes of a warp (running sum passed by shuffle)
+//   M = 16          two such warps chained (the running sum handed on through shared memory)
 //   every other M   replica axis split over the warps of a block (through shared memory), 64
-//                   registers, 1024 threads per SM: SPLIT_R2 two replicas per warp with 128-bit
-//                   accesses up to M = 20 (6.5-6.65 TB/s at M = 5 .. 20; one replica per warp
-//                   measured 5.8-6.2 at M = 5, 6, 7 and 4.4-5.6 beyond), SPLIT_R4 four per warp
-//                   with 64-bit accesses above (6.5 TB/s at M = 24, 32 against 6.1-6.3 for R2:
-//                   blocks of more than 10 warps wait too long at the barrier)
-// The ID names a translation unit: a replica count with its own kernels, one of the split
-// forms, or the first-steps form.
+//                   registers: SPLIT_R2 two replicas per warp with 128-bit accesses up to M = 20
+//                   (6.55-6.8 TB/s at M = 5 .. 20; one replica per warp measured 5.8-6.2 at
+//                   M = 5, 6, 7 and 4.4-5.6 beyond), SPLIT_R4 four per warp with 64-bit accesses
+//                   above (6.5 TB/s at M = 24, 32 against 6.1-6.3 for R2: blocks of more than 10
+//                   warps wait too long at the barrier); two column groups per block where
+//                   that keeps the SM's thread slots filled
+// The ID names a translation unit: a replica count with its own kernels (1, 2, 3, 4, 8, 16), one
+// of the split forms, or the first-steps form.
 enum { SHAPE_FIRST_STEPS = 0, SHAPE_SPLIT_R4 = 1000, SHAPE_SPLIT_R2 = 1002 };
 
 template <int ID, bool Q>
@@ -105,15 +128,16 @@ int launch_outer_shape(int var, int tk, const OuterArgs &a, cudaStream_t s) {
   else if constexpr (ID == 2) return launch_outer_m<Q, 2, 1, 4, 128, 6>(var, tk, a, s);
   else if constexpr (ID == 3) return launch_outer_m<Q, 3, 1, 4, 128, 4>(var, tk, a, s);
   else if constexpr (ID == 4) return launch_outer_m<Q, 4, 2, 4, 256, 4>(var, tk, a, s);
-  // M = 8: 5 resident blocks (96 registers) measured 4 % faster than 4; the quantised eager
-  // form needs ~100 registers and would spill under that cap
-  else if constexpr (ID == 8) return launch_outer_m<Q, 8, 2, 4, 128, Q ? 4 : 5>(var, tk, a, s);
+  // M = 8: blocks of 256 threads (2 KB of every row per block) measured 0.7 % faster than 128
+  else if constexpr (ID == 8) return launch_outer_m<Q, 8, 2, 4, 256, 2>(var, tk, a, s);
+  // M = 16: two M = 8 warps chained per 16 columns, 4 such groups per block (1 KB of every row)
+  else if constexpr (ID == 16) return launch_outer_chain<Q, 2, 256, 2>(var, tk, a, s);
   else if constexpr (ID == SHAPE_SPLIT_R4) return launch_outer_split<Q, 2, 4>(var, tk, a, s);
   else if constexpr (ID == SHAPE_SPLIT_R2) return launch_outer_split<Q, 4, 2>(var, tk, a, s);
   else return launch_outer_first_steps<Q>(var, tk, a, s);
 }
 
 // the translation units
-#define DILOCO_FOR_EACH_SHAPE(X) X(0) X(1) X(2) X(3) X(4) X(8) X(1000) X(1002)
+#define DILOCO_FOR_EACH_SHAPE(X) X(0) X(1) X(2) X(3) X(4) X(8) X(1000) X(1002) X(16)
 
 } // namespace diloco

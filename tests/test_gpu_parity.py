@@ -111,6 +111,17 @@ def test_tensor_map_implementation(oracle, impl, variant, M, P):
     run_outer_steps(oracle, variant, M, P, 0, steps=3, seed=670 + M, impl=impl)
 
 
+@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("theta_kind", [0, 1, 2])
+@pytest.mark.parametrize("P", [150_001, 63, 4_100])
+def test_sixteen_replicas_forms(oracle, variant, theta_kind, P):
+    """M = 16 through its default form (two chained warps per 16 columns, the running sum handed
+    from warp to warp through shared memory and a named barrier) and through both forced
+    warp-split forms: the same ordered sum, the oracle's bits."""
+    for impl in (binding.IMPL_AUTO, binding.IMPL_SPLIT_R2, binding.IMPL_SPLIT_R4):
+        run_outer_steps(oracle, variant, 16, P, theta_kind, steps=2, seed=690 + theta_kind, impl=impl)
+
+
 def test_tensor_map_implementation_large_m_and_fragments(oracle):
     """M = 32 and 64 (narrow tiles only: three stages of wider ones do not fit shared memory and
     the call falls back to the direct form), and a fragment whose base is not at column 0."""
