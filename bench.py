@@ -17,7 +17,8 @@ step through diloco_outer_step_host with the state in pinned host memory (copies
 timed region); `cpu_baseline` is the CPU oracle timed on this machine's host cores; `shapes`
 (default single-GPU run only) holds the same kernel measurements for every other headline
 shape - cfg1, cfg4b, cfg4c, the cfg2 and cfg3 phases, cfg0 cold and warm - each with the
-clock samples of its own timed region.
+clock samples of its own timed region, and `replica_sweep` the eager step at the replica counts
+in between (M = 1 ... 64), one figure per kernel form.
 
 With --impl reference the CPU oracle itself is timed on the same workload (there is no
 reference implementation of this path; the paper ships no code).
@@ -193,6 +194,13 @@ def shard_bounds(P_total: int, world: int, rank: int, quantum: int = 64):
     return lo, hi
 
 
+def workload_of(args, inputs):
+    """The named workload, with its replica count replaced if --M was given (other kernel forms)."""
+    import dataclasses
+    w = inputs.WORKLOADS[args.workload]
+    return dataclasses.replace(w, M=args.M) if getattr(args, "M", 0) else w
+
+
 def config_dict(args, w, P_per_gpu: int) -> dict:
     """What the workload is; the same dict in both arms (GPU path and CPU reference)."""
     phase = w.H > 0 and not args.outer_only
@@ -258,7 +266,7 @@ def run_reference(args):
     import oracle
     from paper_2502_12996_b200 import inputs
     oracle.build()
-    w = inputs.WORKLOADS[args.workload]
+    w = workload_of(args, inputs)
     P_cfg = args.P or w.P
     P = oracle_sample_size(w, P_cfg)
     cores = os.cpu_count() or 1
@@ -296,12 +304,12 @@ def stats(xs):
 class Shape:
     """One workload resident on the device: state, library handle, gradients, and the timed loop."""
 
-    def __init__(self, name, args, dev, rank, world, P=None, phase=None, variant=None, comm="f32"):
+    def __init__(self, name, args, dev, rank, world, P=None, phase=None, variant=None, comm="f32", workload=None):
         import torch
         from paper_2502_12996_b200 import binding, inputs
         self.torch, self.binding, self.inputs = torch, binding, inputs
         self.name, self.dev = name, dev
-        w = self.w = inputs.WORKLOADS[name]
+        w = self.w = workload or inputs.WORKLOADS[name]
         self.P = P or w.P
         if args.strong and P is None:
             lo, hi = shard_bounds(self.P, world, rank)
@@ -567,9 +575,9 @@ def run_ours(args):
     barrier = dist.barrier if world > 1 else None
     peak, peak_kind = load_peak()
     traffic = load_traffic()
-    w = inputs.WORKLOADS[args.workload]
+    w = workload_of(args, inputs)
 
-    main = Shape(args.workload, args, dev, rank, world, P=args.P or None, comm=args.comm)
+    main = Shape(args.workload, args, dev, rank, world, P=args.P or None, comm=args.comm, workload=w)
     ok, why = main.fits()
     if world > 1:                                           # every rank must take the same branch
         t = torch.tensor([0 if ok else 1], device=red_dev)
@@ -701,7 +709,7 @@ def run_ours(args):
 
     # --- the other headline shapes, each measured like the main one, with its own clock record
     shapes = {}
-    if args.shapes and world == 1 and not args.P:
+    if args.shapes and world == 1 and not args.P and not args.M:
         shapes[args.workload] = main_rec
         plan = [("cfg1", None, 10), ("cfg4a", None, 10), ("cfg4b", None, 10), ("cfg4c", None, 10),
                 ("cfg2", True, 3), ("cfg3", True, 3)]
@@ -731,6 +739,23 @@ def run_ours(args):
                               warm_l2={"outer": warm["outer"], "clocks": warm["clocks"],
                                        "l2": "warm: back-to-back launches, state resident in L2; GB/s is not HBM bandwidth"})
         sh.free()
+
+    # --- the eager step at the replica counts between and beyond the configurations' (fp32, 6e8 / M
+    # parameters: about 20 GB of traffic per step), so that every kernel form has a figure in this line
+    sweep = {}
+    if args.shapes and world == 1 and not args.P and not args.M:
+        for M_ in (1, 3, 5, 6, 7, 9, 11, 12, 13, 20, 24, 32, 64):
+            wl = inputs.Workload(f"sweep_M{M_}", 9, M=M_, P=int(6e8 / M_) // 1024 * 1024 + 3, shape_index=M_)
+            sh = Shape(wl.name, args, dev, rank, world, variant=2, workload=wl)
+            if not sh.fits()[0]:
+                continue
+            sh.allocate()
+            r, _, c = sh.measure(flush, sampler, 5, 3)
+            rec = sh.record(r, c, peak, traffic)
+            o = rec["outer"]
+            sweep[str(M_)] = {"P": sh.P, "ms": o["ms"]["mean"], "GBps": o["GBps"], "frac": o["frac"],
+                              "frac_of_nominal_8000": o["frac_of_nominal_8000"], "sm_mhz": c["sm_mhz"], "reasons": c["reasons"]}
+            sh.free()
 
     # --- a plain device copy measured in this run, the same way the recorded peak was
     copy_gbs = None
@@ -771,7 +796,7 @@ def run_ours(args):
                 "dtype": "f32", "data": "synthetic", "config": config_dict(args, w, P),
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
                 "replica_params_per_s": value * M, "copy_gbs_this_run": copy_gbs, "kernels": kernels or None,
-                "shapes": shapes or None}
+                "shapes": shapes or None, "replica_sweep": sweep or None}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -820,6 +845,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--variant", default="eager", choices=list(VARIANTS))
     ap.add_argument("--P", type=int, default=0, help="override the workload's parameter count (per GPU)")
+    ap.add_argument("--M", type=int, default=0, help="override the workload's replica count (1 .. 64)")
     ap.add_argument("--kernel", type=int, default=0, choices=range(len(KERNEL_IMPLS)),
                     help="kernel form, DILOCO_IMPL_*: " + ", ".join(f"{i} {n}" for i, n in enumerate(KERNEL_IMPLS)))
     ap.add_argument("--comm", default="f32", choices=list(COMM),

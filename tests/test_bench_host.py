@@ -42,7 +42,7 @@ def test_both_arms_describe_the_workload_identically():
     import argparse
     from paper_2502_12996_b200 import inputs
     args = argparse.Namespace(workload=bench.DEFAULT_WORKLOAD, variant="eager", outer_only=False, strong=False, kernel=0,
-                              comm="f32")
+                              comm="f32", M=0)
     w = inputs.WORKLOADS[bench.DEFAULT_WORKLOAD]
     cfg = bench.config_dict(args, w, w.P)
     assert cfg["workload"] == "cfg4a" and cfg["M"] == 2 and cfg["P_per_gpu"] == 2_400_000_000
