@@ -420,25 +420,27 @@ class Shape:
         return rows, launches, sampler.window(t0, t1, t_warm)
 
     def record(self, rows, clocks, peak, traffic):
-        """The figures of one shape as they go into the JSON line."""
+        """The figures of one shape as they go into the JSON line (rounded: the line carries many)."""
         w, P = self.w, self.P
         outer_bpp, adam_bpp = self.bytes_per_param()
         outer = stats([r[1] for r in rows])
         vname = [k for k, v in VARIANTS.items() if v == self.variant][0]
-
         in_l2 = state_bytes_per_param(w.M, w.theta_kind) * P <= 4 * L2_BYTES   # ncu's per-index DRAM traffic was
 
         def kernel(name, ms, bpp, key):                                         # captured on HBM-resident sizes
             gbs = bpp * P / (ms["mean"] * 1e-3) / 1e9
             tr = None if in_l2 else traffic.get(key)
-            return {"kernel": name, "ms": ms, "algorithmic_bytes_per_param": bpp, "GBps": gbs, "frac": gbs / peak,
-                    "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS, "GBps_best": bpp * P / (ms["min"] * 1e-3) / 1e9,
-                    "ncu_dram_bytes_per_param": (tr[0] if tr else None), "ncu_profile": (tr[1] if tr else None)}
-        rec = {"M": w.M, "P": P, "theta": THETA_NAMES[w.theta_kind], "state_GB": state_bytes_per_param(w.M, w.theta_kind) * P / 1e9,
-               "step_ms": stats([r[0] for r in rows]), "params_per_s": P / (sum(r[0] for r in rows) / len(rows) * 1e-3),
+            return {"kernel": name, "ms": {k: round(ms[k], 5) for k in ("mean", "median", "min")}, "n": ms["n"],
+                    "algorithmic_bytes_per_param": bpp, "GBps": round(gbs, 1), "frac": round(gbs / peak, 4),
+                    "frac_of_nominal_8000": round(gbs / NOMINAL_HBM_GBS, 4),
+                    "ncu_dram_bytes_per_param": (tr[0] if tr else None)}
+        step = stats([r[0] for r in rows])
+        rec = {"M": w.M, "P": P, "theta": THETA_NAMES[w.theta_kind],
+               "state_GB": round(state_bytes_per_param(w.M, w.theta_kind) * P / 1e9, 2),
+               "step_ms": round(step["mean"], 5), "params_per_s": round(P / (step["mean"] * 1e-3), 1),
                "outer": kernel(f"diloco_outer_{vname}", outer, outer_bpp,
                                ("outer", vname, w.M, w.theta_kind) if not self.comm[0] else None),
-               "clocks": clocks}
+               "clocks": {k: clocks.get(k) for k in ("sm_mhz", "reasons", "power_w_max", "samples")}}
         if self.phase:
             adam = stats([r[2] / w.H for r in rows])
             rec["adamw"] = kernel("diloco_inner_adamw", adam, adam_bpp, ("adamw", "-", w.M, w.theta_kind))
@@ -593,8 +595,8 @@ def run_ours(args):
     main.allocate()
     rows, launches, clocks = main.measure(flush, sampler, args.steps, args.warmup, barrier)
     main_rec = main.record(rows, clocks, peak, traffic)
-    step_ms = main_rec["step_ms"]["mean"]
-    outer_ms = main_rec["outer"]["ms"]["mean"]
+    step_ms = sum(r[0] for r in rows) / len(rows)
+    outer_ms = sum(r[1] for r in rows) / len(rows)
     P, M, phase = main.P, w.M, main.phase
     if world > 1:
         t = torch.tensor([step_ms, outer_ms], device=red_dev, dtype=torch.float64)
@@ -616,10 +618,11 @@ def run_ours(args):
     dom_ms = dom["ms"]["mean"] if dom is not main_rec["outer"] else outer_ms
     achieved = dom["algorithmic_bytes_per_param"] * P / (dom_ms * 1e-3) / 1e9
     tr = dom["ncu_dram_bytes_per_param"]
+    tr_src = traffic.get(("adamw", "-", M, w.theta_kind) if dom is not main_rec["outer"] else ("outer", args.variant, M, w.theta_kind))
     roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                 "algorithmic_bytes_per_param": dom["algorithmic_bytes_per_param"], "traffic": (tr * P if tr else None),
-                "traffic_source": (f"ncu dram bytes per index of {dom['ncu_profile']} x P" if tr else None),
+                "traffic_source": (f"ncu dram bytes per index of {tr_src[1]} x P" if tr and tr_src else None),
                 "kernel_ms": dom_ms, "outer_ms_median": main_rec["outer"]["ms"]["median"],
                 "outer_ms_min": main_rec["outer"]["ms"]["min"]}
     if roofline["frac"] > 1.0:
@@ -753,8 +756,8 @@ def run_ours(args):
             r, _, c = sh.measure(flush, sampler, 5, 3)
             rec = sh.record(r, c, peak, traffic)
             o = rec["outer"]
-            sweep[str(M_)] = {"P": sh.P, "ms": o["ms"]["mean"], "GBps": o["GBps"], "frac": o["frac"],
-                              "frac_of_nominal_8000": o["frac_of_nominal_8000"], "sm_mhz": c["sm_mhz"], "reasons": c["reasons"]}
+            sweep[str(M_)] = {"P": sh.P, "ms": round(o["ms"]["mean"], 4), "GBps": o["GBps"],
+                              "frac_of_nominal_8000": o["frac_of_nominal_8000"], "sm_mhz": c["sm_mhz"]}
             sh.free()
 
     # --- a plain device copy measured in this run, the same way the recorded peak was

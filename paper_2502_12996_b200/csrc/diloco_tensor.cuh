@@ -20,7 +20,7 @@
 //              the group that drained it has finished reading shared memory
 // Same arithmetic, same order, same bits as the direct form.  fp32 theta, M at run time.
 // Measured (eager fp32, GB/s; direct form in brackets): T = 256: M = 2 2548 [6760], M = 4 4401
-// [6773], M = 8 6163-6573 [6729], M = 16 6250 [6554], M = 32 falls back.  One CTA per SM works
+// [6773], M = 8 6163-6573 [6755], M = 16 6250 [6737], M = 32 falls back.  One CTA per SM works
 // through its tiles one after the other, so below M = 8 the per-tile latency of the two passes
 // (about 1 us) is not hidden by anything, and at M = 16 only three 68 KB stages fit, i.e. one
 // tile of loads in flight.  A hybrid with TMA loads and ordinary stores from registers (half the
