@@ -650,6 +650,15 @@ def run_ours(args):
             bpp = outer_bytes_per_param(v, M, w.theta_kind)
             kernels[f"outer_{name}"] = {"ms": ms, "GBps": bpp * P / ms / 1e6, "frac": bpp * P / ms / 1e6 / peak,
                                         "params_per_s": P / ms * 1e3}
+        # the standard step with one shared copy of start and momentum (8 M + 16 B per index in fp32)
+        if w.theta_kind == 0:
+            ss = binding.State(M=M, P=P, stride=stride, theta=st["theta"], start=st["start"][0], outer_mom=st["outer_mom"][0],
+                               shared_outer_state=True)
+            ms = time_kernel(lambda: ss.outer_standard())
+            bpp = 8 * M + 16
+            kernels["outer_standard_shared_state"] = {"ms": ms, "GBps": bpp * P / ms / 1e6, "frac": bpp * P / ms / 1e6 / peak,
+                                                      "params_per_s": P / ms * 1e3}
+            ss.close()
         # the worker form: one replica, Delta_m sent / summed Delta received (40 B per index in fp32)
         if w.theta_kind == 0:
             sw = binding.State(M=1, P=P, stride=stride, theta=st["theta"][0], start=st["start"][0],

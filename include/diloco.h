@@ -118,19 +118,29 @@ typedef struct {
                            line 11 with t-H replaced by t-DH,
                              g_m = (Delta_m^(t) - Delta_m^(t-DH)) / M + Delta^(t-DH).
                            At most DILOCO_MAX_OVERLAP. */
+  int32_t shared_outer_state; /* 0: start and outer_mom are [M, stride], one copy per replica (every call works).
+                           1: standard DiLoCo only: under Algorithm 1 every replica's OuterOpt sees the same
+                           start point and the same gradient, so the M copies of s_m and b_m stay bit-identical
+                           for ever; with this flag the state keeps ONE copy, start and outer_mom are [stride],
+                           and the standard step moves 8 M + 16 bytes per index instead of 24 M (same bits in
+                           theta).  diloco_outer_standard, diloco_outer_fragment(_step) with variant 0 and
+                           diloco_inner_adamw work; every other outer call returns DILOCO_ERR_BAD_STATE (the
+                           delayed and eager steps let the replicas' start points differ). */
 } diloco_config_t;
 
 typedef struct {
   void *theta;             /* [M, stride] fp32 or bf16 per theta_kind: theta_m^(t)                      */
   float *master;           /* [M, stride] fp32, only for DILOCO_THETA_MASTER_BF16, else NULL            */
-  float *start;            /* [M, stride] fp32: s_m = theta_m^(t-H)                 (Alg. 1-3 line 7)   */
+  float *start;            /* [M, stride] fp32: s_m = theta_m^(t-H)                 (Alg. 1-3 line 7);
+                              [stride] with shared_outer_state                                            */
   float *delta_prev_local; /* [D, M, stride] fp32, D = overlap_steps: Delta_m of the last D outer steps, a
                               ring indexed by (outer-step counter mod D): the step that reads a generation
                               overwrites it.  Eager only, else may be NULL              (Alg. 3 l.11)    */
   float *delta_prev_avg;   /* [D, stride] fp32: the means of those steps, i.e. the all-reduces in flight;
                               delayed and eager, may be NULL if only the standard step is used
                                                                                     (Alg. 2-3 line 10)  */
-  float *outer_mom;        /* [M, stride] fp32: b_m, Nesterov buffer of OuterOpt                        */
+  float *outer_mom;        /* [M, stride] fp32: b_m, Nesterov buffer of OuterOpt; [stride] with
+                              shared_outer_state                                                          */
   float *adam_m;           /* [M, stride] fp32 first moment;  NULL if diloco_inner_adamw is not used    */
   float *adam_v;           /* [M, stride] fp32 second moment; NULL if diloco_inner_adamw is not used    */
   uint32_t *device_status; /* 1 word, zero-initialised by the caller; needed only by DILOCO_IMPL_BULK,

@@ -30,7 +30,8 @@ class Config(ctypes.Structure):
                 ("outer_lr", ctypes.c_float), ("outer_momentum", ctypes.c_float),
                 ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
                 ("weight_decay", ctypes.c_float), ("theta_kind", ctypes.c_int32), ("grad_kind", ctypes.c_int32),
-                ("have_prev", ctypes.c_int32), ("impl", ctypes.c_int32), ("overlap_steps", ctypes.c_int32)]
+                ("have_prev", ctypes.c_int32), ("impl", ctypes.c_int32), ("overlap_steps", ctypes.c_int32),
+                ("shared_outer_state", ctypes.c_int32)]
 
 
 class Buffers(ctypes.Structure):
@@ -189,14 +190,14 @@ class State:
                  delta_prev_avg=None, adam_m=None, adam_v=None, device_status=None, comm_scratch=None, H=0,
                  outer_lr=0.7,
                  outer_momentum=0.9, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1, theta_kind=THETA_F32,
-                 grad_kind=GRAD_F32, have_prev=None, impl=IMPL_AUTO, overlap_steps=1):
+                 grad_kind=GRAD_F32, have_prev=None, impl=IMPL_AUTO, overlap_steps=1, shared_outer_state=False):
         self._handle = ctypes.c_void_p()
         self.tensors = dict(theta=theta, master=master, start=start, delta_prev_local=delta_prev_local,
                             delta_prev_avg=delta_prev_avg, outer_mom=outer_mom, adam_m=adam_m, adam_v=adam_v,
                             device_status=device_status, comm_scratch=comm_scratch)
         have_prev = overlap_steps if have_prev is None else int(have_prev)      # default: every generation seeded
         self.config = Config(M, H, P, stride, outer_lr, outer_momentum, beta1, beta2, eps, weight_decay,
-                             theta_kind, grad_kind, have_prev, impl, overlap_steps)
+                             theta_kind, grad_kind, have_prev, impl, overlap_steps, int(bool(shared_outer_state)))
         self.buffers = make_buffers(**self.tensors)
         _check(load_library().diloco_state_init(ctypes.byref(self.config), ctypes.byref(self.buffers),
                                                 ctypes.byref(self._handle)), "diloco_state_init")

@@ -91,6 +91,7 @@ int validate_config(const diloco_config_t *c) {
   if (c->overlap_steps < 1) return DILOCO_ERR_INVALID_ARG;
   if (c->overlap_steps > DILOCO_MAX_OVERLAP) return DILOCO_ERR_UNSUPPORTED;
   if (c->have_prev < 0 || c->have_prev > c->overlap_steps) return DILOCO_ERR_INVALID_ARG;
+  if (c->shared_outer_state != 0 && c->shared_outer_state != 1) return DILOCO_ERR_INVALID_ARG;
   // 128-byte rows for every dtype in use
   if ((c->stride * 4) % 128 != 0) return DILOCO_ERR_MISALIGNED;
   if (c->theta_kind != DILOCO_THETA_F32 && (c->stride * 2) % 128 != 0) return DILOCO_ERR_MISALIGNED;
@@ -195,6 +196,8 @@ int check_variant(const diloco_state *st, int var) {
   if (var < VAR_STANDARD || var > VAR_EAGER) return DILOCO_ERR_INVALID_ARG;
   int rc = check_device(st);
   if (rc != DILOCO_OK) return rc;
+  // one shared copy of s and b exists only for the standard step: the others let the replicas' copies differ
+  if (st->cfg.shared_outer_state && var != VAR_STANDARD) return DILOCO_ERR_BAD_STATE;
   if (var != VAR_STANDARD && !st->buf.delta_prev_avg) return DILOCO_ERR_BAD_STATE;
   if (var == VAR_EAGER && !st->buf.delta_prev_local) return DILOCO_ERR_BAD_STATE;
   return DILOCO_OK;
@@ -386,8 +389,28 @@ int launch_tensor(const diloco_state *st, int var, const OuterArgs &a, cudaStrea
   return launch_tensor_t<VAR_EAGER, T>(st, a, s);
 }
 
+template <int TK>
+int launch_standard_shared_t(const OuterArgs &a, cudaStream_t s) {
+  constexpr int NT = 256;
+  long long blocks = (a.P / 4 + NT - 1) / NT;
+  if (blocks < 1) blocks = 1; // the last block also handles the P % 4 tail
+  if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
+  outer_standard_shared_kernel<TK, NT><<<(unsigned)blocks, NT, 0, s>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1);
+  return DILOCO_OK;
+}
+
 int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t len, cudaStream_t s, int ring = -1) {
   OuterArgs a = outer_args(st, offset, len, ring);
+  if (st->cfg.shared_outer_state) { // check_variant has let only the standard step through
+    switch (st->cfg.theta_kind) {
+      case TK_F32: return launch_standard_shared_t<TK_F32>(a, s);
+      case TK_BF16: return launch_standard_shared_t<TK_BF16>(a, s);
+      default: return launch_standard_shared_t<TK_MASTER_BF16>(a, s);
+    }
+  }
   // The tensor form: fp32 theta, needs the status word for its bounded waits; falls back to the
   // direct form where a stage ring of three tiles does not fit shared memory.
   if (st->cfg.impl >= DILOCO_IMPL_TENSOR_T256 && st->cfg.impl <= DILOCO_IMPL_TENSOR_T64 && !boot &&
@@ -655,6 +678,7 @@ int diloco_outer_quantized(diloco_state_t *st, int32_t variant, int32_t comm_for
   if (rc != DILOCO_OK) return rc;
   if (comm_format == DILOCO_COMM_F32) return outer_whole(st, variant, stream);
   if (comm_format != DILOCO_COMM_BF16 && comm_format != DILOCO_COMM_EXMY) return DILOCO_ERR_INVALID_ARG;
+  if (st->cfg.shared_outer_state) return DILOCO_ERR_BAD_STATE; // the wire formats have per-replica kernels only
   if (comm_format == DILOCO_COMM_EXMY) {
     if (exp_bits < 1 || exp_bits > 5 || man_bits < 0 || exp_bits + man_bits > 7) return DILOCO_ERR_INVALID_ARG;
     if (!st->buf.comm_scratch) return DILOCO_ERR_BAD_STATE;
@@ -679,6 +703,7 @@ int diloco_outer_quantized_static(diloco_state_t *st, int32_t variant, int32_t c
   // words, the check keeps that true if the state limit is ever raised
   if (st->cfg.M > kStaticScratchWords) return DILOCO_ERR_UNSUPPORTED;
   if (comm_format == DILOCO_COMM_F32) return outer_whole(st, variant, stream);
+  if (st->cfg.shared_outer_state) return DILOCO_ERR_BAD_STATE;
   unsigned *scratch = nullptr; // only the EXMY formats reduce maxima; the others never touch the array
   if (comm_format == DILOCO_COMM_EXMY) {
     // check_variant has verified that the state's GPU is the current one
@@ -857,6 +882,7 @@ int diloco_outer_fragment_step_quantized(diloco_state_t *st, int32_t variant, in
   if (rc != DILOCO_OK) return rc;
   if (fragment_id < 0 || (size_t)fragment_id >= st->frags.size()) return DILOCO_ERR_INVALID_ARG;
   if (comm_format != DILOCO_COMM_BF16 && comm_format != DILOCO_COMM_EXMY) return DILOCO_ERR_INVALID_ARG;
+  if (st->cfg.shared_outer_state) return DILOCO_ERR_BAD_STATE;
   if (comm_format == DILOCO_COMM_EXMY) {
     if (!valid_exmy(exp_bits, man_bits)) return DILOCO_ERR_INVALID_ARG;
     if (!st->buf.comm_scratch) return DILOCO_ERR_BAD_STATE;
@@ -893,6 +919,7 @@ int diloco_outer_step_host(diloco_state_t *st, int32_t variant, const diloco_buf
   int rc = check_variant(st, variant);
   if (rc != DILOCO_OK) return rc;
   if (chunk < 64 || chunk % 64 != 0) return DILOCO_ERR_INVALID_ARG;
+  if (st->cfg.shared_outer_state) return DILOCO_ERR_BAD_STATE; // the copy plan below assumes one row per replica
   cudaStream_t s_in = static_cast<cudaStream_t>(streams[0]);
   cudaStream_t s_k = static_cast<cudaStream_t>(streams[1]);
   cudaStream_t s_out = static_cast<cudaStream_t>(streams[2]);

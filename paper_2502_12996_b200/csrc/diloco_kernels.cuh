@@ -486,6 +486,54 @@ __global__ void __launch_bounds__(NT, 4) outer_first_steps_kernel(const OuterArg
   }
 }
 
+// ---------------------------------------------------------------- standard step, one shared copy of s and b
+// Algorithm 1 with the outer parameters and the momentum stored once instead of once per replica
+// (under the standard step the M copies are bit-identical for ever: same start, same gradient).
+// Per index: reads s, b and the M theta_m, writes s, b and the M theta_m: 8 M + 16 bytes instead
+// of 24 M.  One column of V indices per thread, M at run time; the theta_m are loaded four at a
+// time so that a thread keeps 4 vectors in flight, and summed in the order m = 0 .. M-1.
+template <int TK, int V>
+__device__ __forceinline__ void standard_shared_column(const OuterArgs &a, long long i) {
+  float s[V], b[V], acc[V];
+  F32Vec<V>::load(a.start + i, s);
+  F32Vec<V>::load(a.mom + i, b);
+  for (int m0 = 0; m0 < a.M; m0 += 4) {
+    float x[4][V];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+      if (m0 + r < a.M) load_theta<TK, V>(a, (m0 + r) * a.stride + i, x[r]);
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+      if (m0 + r < a.M) {
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          const float d = s[e] - x[r][e];                  // Alg. 1 line 7
+          acc[e] = (m0 + r == 0) ? d : acc[e] + d;         // line 8, replica order
+        }
+      }
+  }
+#pragma unroll
+  for (int e = 0; e < V; ++e) {
+    const float mean = acc[e] / a.fM;
+    nesterov(mean, a.eta, a.mu, b[e], s[e]);               // line 10, once for all replicas
+  }
+  F32Vec<V>::store(a.mom + i, b);
+  F32Vec<V>::store(a.start + i, s);
+  for (int m = 0; m < a.M; ++m) store_theta<TK, V>(a, m * a.stride + i, s);
+}
+
+template <int TK, int NT>
+__global__ void __launch_bounds__(NT, 4) outer_standard_shared_kernel(const OuterArgs a) {
+  constexpr int V = 4;
+  const long long nvec = a.P / V;
+  const long long j = (long long)blockIdx.x * NT + threadIdx.x;
+  if (j < nvec) standard_shared_column<TK, V>(a, j * V);
+  if (blockIdx.x == gridDim.x - 1) {
+    const long long i = nvec * V + threadIdx.x;
+    if (i < a.P) standard_shared_column<TK, 1>(a, i);
+  }
+}
+
 // ---------------------------------------------------------------- outer step, M = 8 W: a chain of W warps
 // The lane-split shape of M = 8 (two half-warps of 16 columns, 4 replicas per lane, 128-bit
 // accesses, no shared-memory exchange of the contributions) extended to M = 16, 24, 32: W warps

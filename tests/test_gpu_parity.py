@@ -184,6 +184,50 @@ def test_bounded_device_wait_runs_out_and_is_reported(oracle, M, P, impl):
     state.close()
 
 
+@pytest.mark.parametrize("theta_kind", [0, 1, 2])
+@pytest.mark.parametrize("M,P", [(1, 9_001), (2, 300_003), (4, 200_005), (5, 70_001), (8, 50_002), (16, 20_003), (64, 3_001),
+                                 (3, 2)])
+def test_standard_step_with_one_shared_copy_of_the_outer_state(oracle, theta_kind, M, P):
+    """Algorithm 1 with start and outer_mom stored once ([stride]) instead of once per replica:
+    theta and the shared copy must equal EVERY replica's row of the per-replica oracle, bit for
+    bit, over several steps; every other outer call refuses such a state."""
+    st, checks = make(M, P, 720 + M, theta_kind)
+    h = host_copy(st)                                          # per-replica oracle: all M rows start equal
+    h["outer_mom"][:] = h["outer_mom"][0]
+    shared = dict(st)
+    shared["start"] = st["start"][0].clone()
+    shared["outer_mom"] = st["outer_mom"][0].clone()
+    state = binding.State.from_dict(shared, shared_outer_state=True)
+    for k in range(3):
+        if k:
+            inputs.inner_phase_standin(st)                     # theta_m <- start_m + noise; the rows of start are stale here,
+            for key in ("theta", "master"):                    # so rebuild theta from the shared copy instead
+                if st.get(key) is not None:
+                    noise = st[key][:, :P].float() - st["start"][:, :P]
+                    st[key][:, :P] = (shared["start"][:P] + noise).to(st[key].dtype)
+            h["theta"], h["master"] = to_numpy(st["theta"]), to_numpy(st["master"])
+        state.outer_standard()
+        oracle_outer(oracle, 0, h, M, P, st["stride"], 0.7, 0.9, theta_kind)
+        torch.cuda.synchronize()
+        got = dict(theta=st["theta"], master=st["master"])
+        assert_state_equal(got, h, keys=("theta", "master"), what=f"shared standard M={M} kind={theta_kind} step {k + 1}")
+        for m in range(M):
+            for key in ("start", "outer_mom"):
+                one = {key: shared[key][:P]}
+                assert_state_equal(one, {key: h[key][m, :P]}, keys=(key,), what=f"shared {key} vs replica {m}")
+    assert float(shared["start"][P:].min()) == 3.0 and float(shared["outer_mom"][P:].max()) == 3.0   # padding untouched
+    for c in checks:
+        c()
+    for call in (state.outer_eager, state.outer_delayed, lambda: state.outer_quantized(0, binding.COMM_BF16)):
+        with pytest.raises(binding.DilocoError) as e:
+            call()
+        assert e.value.status == binding.ERR_BAD_STATE
+    state.fragments_set([0], [min(P, 64)])
+    state.outer_fragment_step(binding.STANDARD, 0)
+    torch.cuda.synchronize()
+    state.close()
+
+
 @pytest.mark.parametrize("eta,mu", [(0.4, 0.9), (1.0, 0.0), (0.7, 0.0)])
 def test_other_outer_hyperparameters(oracle, eta, mu):
     run_outer_steps(oracle, 2, 4, 65_537, 0, steps=3, seed=700, eta=eta, mu=mu)
