@@ -718,7 +718,7 @@ def run_ours(args):
         if pick == args.workload:
             e2e = run_e2e(main, args, world, dist, red_dev, max(3, min(args.steps, 10 if main.P < 2e8 else 3)))
             if e2e.get("value") is None and world == 1 and not args.P and args.workload != "cfg1":
-                first_error, e2e, e2e_shape = e2e.get("error"), None, "cfg1"   # page-locking failed: a small shape instead
+                e2e, e2e_shape = None, "cfg1"                 # page-locking failed: a small shape instead
         elif pick is not None:
             e2e_shape = pick                                   # measured below, once the main state is freed
         else:
