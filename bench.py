@@ -879,7 +879,8 @@ def main():
                     help="kernel form, DILOCO_IMPL_*: " + ", ".join(f"{i} {n}" for i, n in enumerate(KERNEL_IMPLS)))
     ap.add_argument("--comm", default="f32", choices=list(COMM),
                     help="wire format of the outer gradients (quantised communication)")
-    ap.add_argument("--chunk", type=int, default=64 * 16384, help="elements per chunk of the host-buffer path")
+    ap.add_argument("--chunk", type=int, default=64 * 65536,
+                    help="elements per chunk of the host-buffer path (4 Mi: 16 MB copies measured 7 %% faster than 4 MB ones)")
     ap.add_argument("--e2e-host-fraction", type=float, default=0.5,
                     help="share of the host's available memory that the end-to-end leg may page-lock")
     ap.add_argument("--strong", action="store_true", help="split the workload's P across ranks instead of one full shape per rank")
