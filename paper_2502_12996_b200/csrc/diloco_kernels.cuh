@@ -392,9 +392,11 @@ __device__ __forceinline__ void outer_column(const OuterArgs &a, long long i, in
   if (VAR != VAR_STANDARD && m0 == 0) F32Vec<V>::store(a.dpa + i, mean);
 }
 
-// ---------------------------------------------------------------- outer step, runtime M
+// ---------------------------------------------------------------- outer step, runtime M, one thread per column
 // Two sweeps over the replicas: the first forms the mean, the second re-reads s_m and
 // theta_m (L1/L2 hits: the same thread read them a few hundred cycles earlier) and updates.
+// Serves the recording-only first steps (BOOT) of every M and the ragged last P % V indices of
+// every kernel; the steady-state steps have the faster forms above and below.
 template <int VAR, int TK, bool BOOT, int V, bool Q = false>
 __device__ __forceinline__ void outer_column_rt(const OuterArgs &a, long long i) {
   float mean[V];

@@ -802,8 +802,8 @@ def test_bench_line_has_every_contract_key():
 def test_random_configurations(oracle, case):
     """Seeded random (M, P, variant, storage, overlap, wire format, seeded generations): every
     replica count from 1 to 64 lands on one of the kernel forms (per-thread, lane split, warp
-    split, warp per replica, two sweeps), and every combination must equal the oracle bit for
-    bit over several outer steps."""
+    chain, warp split with one or two column groups per block, first-steps form), and every
+    combination must equal the oracle bit for bit over several outer steps."""
     rng = np.random.default_rng(31_000 + case)
     M = int(rng.choice([int(rng.integers(1, 65)), int(rng.choice([12, 20, 24, 28, 36, 40, 44, 48, 52, 56, 60, 64])),
                         int(rng.choice([5, 6, 7, 9, 11, 13, 17, 31, 33, 63]))]))
