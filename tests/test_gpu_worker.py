@@ -174,13 +174,17 @@ def _free_port():
         return s.getsockname()[1]
 
 
-def _rank_main(rank, world, port, variant, D, P, H, phases, theta_kind, out_dir, wire=None):
+def _rank_main(rank, world, port, variant, D, P, H, phases, theta_kind, out_dir, wire=None, backend="gloo"):
     import torch.distributed as dist
     sys.path.insert(0, str(ROOT))
     from paper_2502_12996_b200 import inputs as inp, worker
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
-    dist.init_process_group("gloo", rank=rank, world_size=world)
     torch.cuda.set_device(0)
+    if backend == "nccl":
+        os.environ["NCCL_NVLS_ENABLE"] = "0"
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", 0))
+    else:
+        dist.init_process_group("gloo", rank=rank, world_size=world)
     # every rank draws the same M-replica state from the same seed and keeps its own replica
     st = inp.make_outer_state(world, P, 777, device="cuda:0", theta_kind=theta_kind, with_adam=True, overlap_steps=D)
     stride = st["stride"]
@@ -203,12 +207,17 @@ def _rank_main(rank, world, port, variant, D, P, H, phases, theta_kind, out_dir,
     dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("variant,D,theta_kind,wire", [(2, 1, 0, None), (2, 2, 1, None), (1, 1, 0, None), (0, 1, 0, None),
-                                                       (2, 1, 0, (4, 3)), (2, 2, 1, (2, 1)), (0, 1, 0, (3, 0))])
-def test_two_worker_processes_with_async_all_reduce(oracle, tmp_path, variant, D, theta_kind, wire):
+@pytest.mark.parametrize("variant,D,theta_kind,wire,world,backend",
+                         [(2, 1, 0, None, 2, "gloo"), (2, 2, 1, None, 2, "gloo"), (1, 1, 0, None, 2, "gloo"),
+                          (0, 1, 0, None, 2, "gloo"), (2, 1, 0, (4, 3), 2, "gloo"), (2, 2, 1, (2, 1), 2, "gloo"),
+                          (0, 1, 0, (3, 0), 2, "gloo"),
+                          # one rank over NCCL: the collectives are trivial, but the Worker's asynchronous
+                          # all-reduce / all-gather handles and their stream ordering are NCCL's
+                          (2, 1, 0, None, 1, "nccl"), (2, 2, 0, (4, 3), 1, "nccl"), (0, 1, 1, None, 1, "nccl")])
+def test_worker_processes_with_async_collectives(oracle, tmp_path, variant, D, theta_kind, wire, world, backend):
     import torch.multiprocessing as mp
-    world, P, H, phases = 2, 60_001, 3, 2 * D + 2
-    mp.spawn(_rank_main, args=(world, _free_port(), variant, D, P, H, phases, theta_kind, str(tmp_path), wire),
+    P, H, phases = 60_001, 3, 2 * D + 2
+    mp.spawn(_rank_main, args=(world, _free_port(), variant, D, P, H, phases, theta_kind, str(tmp_path), wire, backend),
              nprocs=world, join=True)
     comm_kw = {} if wire is None else dict(comm=oracle.COMM_EXMY, exp_bits=wire[0], man_bits=wire[1])
     # the same run through the fused oracle
