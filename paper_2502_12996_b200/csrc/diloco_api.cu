@@ -389,17 +389,22 @@ int launch_tensor(const diloco_state *st, int var, const OuterArgs &a, cudaStrea
   return launch_tensor_t<VAR_EAGER, T>(st, a, s);
 }
 
-template <int TK>
-int launch_standard_shared_t(const OuterArgs &a, cudaStream_t s) {
+template <int TK, int U>
+int launch_standard_shared_u(const OuterArgs &a, cudaStream_t s) {
   constexpr int NT = 256;
-  long long blocks = (a.P / 4 + NT - 1) / NT;
+  long long blocks = (a.P / 4 + (long long)NT * U - 1) / ((long long)NT * U);
   if (blocks < 1) blocks = 1; // the last block also handles the P % 4 tail
   if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
-  outer_standard_shared_kernel<TK, NT><<<(unsigned)blocks, NT, 0, s>>>(a);
+  outer_standard_shared_kernel<TK, NT, U><<<(unsigned)blocks, NT, 0, s>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1);
   return DILOCO_OK;
+}
+
+template <int TK>
+int launch_standard_shared_t(const OuterArgs &a, cudaStream_t s) {
+  return a.M <= 4 ? launch_standard_shared_u<TK, 2>(a, s) : launch_standard_shared_u<TK, 1>(a, s);
 }
 
 int launch_outer(diloco_state *st, int var, bool boot, int64_t offset, int64_t len, cudaStream_t s, int ring = -1) {

@@ -492,47 +492,78 @@ __global__ void __launch_bounds__(NT, 4) outer_first_steps_kernel(const OuterArg
 // Algorithm 1 with the outer parameters and the momentum stored once instead of once per replica
 // (under the standard step the M copies are bit-identical for ever: same start, same gradient).
 // Per index: reads s, b and the M theta_m, writes s, b and the M theta_m: 8 M + 16 bytes instead
-// of 24 M.  One column of V indices per thread, M at run time; the theta_m are loaded four at a
-// time so that a thread keeps 4 vectors in flight, and summed in the order m = 0 .. M-1.
-template <int TK, int V>
-__device__ __forceinline__ void standard_shared_column(const OuterArgs &a, long long i) {
-  float s[V], b[V], acc[V];
-  F32Vec<V>::load(a.start + i, s);
-  F32Vec<V>::load(a.mom + i, b);
-  for (int m0 = 0; m0 < a.M; m0 += 4) {
-    float x[4][V];
+// of 24 M.  M at run time; the theta_m are loaded four at a time, all loads of a batch before
+// the first use, and summed in the order m = 0 .. M-1.
+template <int TK, int V, int U>
+__device__ __forceinline__ void standard_shared_columns(const OuterArgs &a, const long long (&idx)[U]) {
+  float s[U][V], b[U][V], acc[U][V];
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
-      if (m0 + r < a.M) load_theta<TK, V>(a, (m0 + r) * a.stride + i, x[r]);
+  for (int u = 0; u < U; ++u) {
+    F32Vec<V>::load(a.start + idx[u], s[u]);
+    F32Vec<V>::load(a.mom + idx[u], b[u]);
+  }
+  for (int m0 = 0; m0 < a.M; m0 += 4) {
+    float x[4][U][V];
 #pragma unroll
     for (int r = 0; r < 4; ++r)
       if (m0 + r < a.M) {
 #pragma unroll
-        for (int e = 0; e < V; ++e) {
-          const float d = s[e] - x[r][e];                  // Alg. 1 line 7
-          acc[e] = (m0 + r == 0) ? d : acc[e] + d;         // line 8, replica order
-        }
+        for (int u = 0; u < U; ++u) load_theta<TK, V>(a, (m0 + r) * a.stride + idx[u], x[r][u]);
+      }
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+      if (m0 + r < a.M) {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+          for (int e = 0; e < V; ++e) {
+            const float d = s[u][e] - x[r][u][e];                     // Alg. 1 line 7
+            acc[u][e] = (m0 + r == 0) ? d : acc[u][e] + d;            // line 8, replica order
+          }
       }
   }
 #pragma unroll
-  for (int e = 0; e < V; ++e) {
-    const float mean = acc[e] / a.fM;
-    nesterov(mean, a.eta, a.mu, b[e], s[e]);               // line 10, once for all replicas
+  for (int u = 0; u < U; ++u) {
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      const float mean = acc[u][e] / a.fM;
+      nesterov(mean, a.eta, a.mu, b[u][e], s[u][e]);                  // line 10, once for all replicas
+    }
+    F32Vec<V>::store(a.mom + idx[u], b[u]);
+    F32Vec<V>::store(a.start + idx[u], s[u]);
   }
-  F32Vec<V>::store(a.mom + i, b);
-  F32Vec<V>::store(a.start + i, s);
-  for (int m = 0; m < a.M; ++m) store_theta<TK, V>(a, m * a.stride + i, s);
+  for (int m = 0; m < a.M; ++m)
+#pragma unroll
+    for (int u = 0; u < U; ++u) store_theta<TK, V>(a, m * a.stride + idx[u], s[u]);
 }
 
-template <int TK, int NT>
-__global__ void __launch_bounds__(NT, 4) outer_standard_shared_kernel(const OuterArgs a) {
+// U columns per thread (columns j, j + NT, ...): with few replicas one column is only 2 + M
+// vectors in flight per thread, too few to keep the memory system busy (M = 2: 6.2 TB/s).
+template <int TK, int NT, int U>
+__global__ void __launch_bounds__(NT, U == 1 ? 4 : 3) outer_standard_shared_kernel(const OuterArgs a) {
   constexpr int V = 4;
   const long long nvec = a.P / V;
-  const long long j = (long long)blockIdx.x * NT + threadIdx.x;
-  if (j < nvec) standard_shared_column<TK, V>(a, j * V);
+  const long long j0 = (long long)blockIdx.x * (NT * U) + threadIdx.x;
+  if (j0 + (long long)(U - 1) * NT < nvec) {
+    long long idx[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) idx[u] = (j0 + (long long)u * NT) * V;
+    standard_shared_columns<TK, V, U>(a, idx);
+  } else {
+    for (int u = 0; u < U; ++u) {
+      const long long j = j0 + (long long)u * NT;
+      if (j < nvec) {
+        const long long one[1] = {j * V};
+        standard_shared_columns<TK, V, 1>(a, one);
+      }
+    }
+  }
   if (blockIdx.x == gridDim.x - 1) {
     const long long i = nvec * V + threadIdx.x;
-    if (i < a.P) standard_shared_column<TK, 1>(a, i);
+    if (i < a.P) {
+      const long long one[1] = {i};
+      standard_shared_columns<TK, 1, 1>(a, one);
+    }
   }
 }
 
