@@ -144,7 +144,8 @@ int validate_buffers(const diloco_config_t *c, const diloco_buffers_t *b) {
 int split_shape_for(int M, int forced) {
   if (forced == DILOCO_IMPL_SPLIT_R2 && M <= 32) return SHAPE_SPLIT_R2; // 16 warps per block at most
   if (forced == DILOCO_IMPL_SPLIT_R4) return SHAPE_SPLIT_R4;
-  return M <= 20 ? SHAPE_SPLIT_R2 : SHAPE_SPLIT_R4;
+  if (M <= 20) return SHAPE_SPLIT_R2;
+  return M <= 48 ? SHAPE_SPLIT_R4 : SHAPE_SPLIT_R8;
 }
 
 template <bool Q>
@@ -165,6 +166,7 @@ int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterA
   }
   switch (split_shape_for(M, impl)) {
     case SHAPE_SPLIT_R2: return launch_outer_shape<SHAPE_SPLIT_R2, Q>(var, tk, a, s);
+    case SHAPE_SPLIT_R8: return launch_outer_shape<SHAPE_SPLIT_R8, Q>(var, tk, a, s);
     default: return launch_outer_shape<SHAPE_SPLIT_R4, Q>(var, tk, a, s);
   }
 }

@@ -59,8 +59,9 @@ int launch_outer_m(int var, int tk, const OuterArgs &a, cudaStream_t s) {
 template <bool Q, int V, int R>
 int launch_outer_split(int var, int tk, const OuterArgs &a, cudaStream_t s) {
   const int warps = (a.M + R - 1) / R;
-  if (warps > 16) return DILOCO_ERR_UNSUPPORTED;
-  const int groups = (warps <= 5 || warps == 8) ? 2 : 1; // 2 x 6 or 2 x 7 warps leave a quarter of the SM's thread slots empty
+  if (warps > (R <= 4 ? 16 : 8)) return DILOCO_ERR_UNSUPPORTED;
+  // 2 x 6 or 2 x 7 warps leave a quarter of the SM's thread slots empty; R = 8 blocks are register-bound
+  const int groups = (R <= 4 && (warps <= 5 || warps == 8)) ? 2 : 1;
   long long blocks = ((a.P / V + 31) / 32 + groups - 1) / groups;
   if (blocks < 1) blocks = 1; // the last block also handles the P % V tail
   if (blocks > 0x7fffffffLL) return DILOCO_ERR_UNSUPPORTED;
@@ -116,11 +117,12 @@ int launch_outer_first_steps(int var, int tk, const OuterArgs &a, cudaStream_t s
 //                   (6.55-6.8 TB/s at M = 5 .. 20; one replica per warp measured 5.8-6.2 at
 //                   M = 5, 6, 7 and 4.4-5.6 beyond), SPLIT_R4 four per warp with 64-bit accesses
 //                   above (6.5 TB/s at M = 24, 32 against 6.1-6.3 for R2: blocks of more than 10
-//                   warps wait too long at the barrier); two column groups per block where
-//                   that keeps the SM's thread slots filled
+//                   warps wait too long at the barrier), SPLIT_R8 eight per warp above M = 48
+//                   (M = 64: 6.44 against 5.9 TB/s, blocks of 8 warps instead of 16); two column
+//                   groups per block where that keeps the SM's thread slots filled
 // The ID names a translation unit: a replica count with its own kernels (1, 2, 3, 4, 8, 16), one
 // of the split forms, or the first-steps form.
-enum { SHAPE_FIRST_STEPS = 0, SHAPE_SPLIT_R4 = 1000, SHAPE_SPLIT_R2 = 1002 };
+enum { SHAPE_FIRST_STEPS = 0, SHAPE_SPLIT_R4 = 1000, SHAPE_SPLIT_R2 = 1002, SHAPE_SPLIT_R8 = 1003 };
 
 template <int ID, bool Q>
 int launch_outer_shape(int var, int tk, const OuterArgs &a, cudaStream_t s) {
@@ -134,10 +136,11 @@ int launch_outer_shape(int var, int tk, const OuterArgs &a, cudaStream_t s) {
   else if constexpr (ID == 16) return launch_outer_chain<Q, 2, 256, 2>(var, tk, a, s);
   else if constexpr (ID == SHAPE_SPLIT_R4) return launch_outer_split<Q, 2, 4>(var, tk, a, s);
   else if constexpr (ID == SHAPE_SPLIT_R2) return launch_outer_split<Q, 4, 2>(var, tk, a, s);
+  else if constexpr (ID == SHAPE_SPLIT_R8) return launch_outer_split<Q, 2, 8>(var, tk, a, s);
   else return launch_outer_first_steps<Q>(var, tk, a, s);
 }
 
 // the translation units
-#define DILOCO_FOR_EACH_SHAPE(X) X(0) X(1) X(2) X(3) X(4) X(8) X(1000) X(1002) X(16)
+#define DILOCO_FOR_EACH_SHAPE(X) X(0) X(1) X(2) X(3) X(4) X(8) X(1000) X(1002) X(1003) X(16)
 
 } // namespace diloco
