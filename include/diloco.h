@@ -40,6 +40,12 @@
  *     IEEE division and square root; the sum over replicas runs m = 0 .. M-1 in order; 1/M
  *     is a division by (float)M.  bf16 is a storage type only (round-to-nearest-even).
  *   - a state is not thread-safe: one caller at a time.
+ *   - CUDA graphs: a steady-state diloco_outer_standard / _delayed / _eager call (have_prev =
+ *     overlap_steps = 1, direct kernels) is one launch whose arguments do not change from step to
+ *     step and may be captured and replayed; the counters advance when the call is captured, not
+ *     when the graph runs.  Do not capture diloco_inner_adamw (its bias corrections are launch
+ *     arguments computed from the step count), steps with overlap_steps > 1 (the ring slot is a
+ *     launch argument) or first steps.  Nothing is said here about the other entry points.
  */
 #ifndef DILOCO_H_
 #define DILOCO_H_

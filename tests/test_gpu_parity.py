@@ -728,6 +728,35 @@ def test_launch_counter():
     torch.cuda.synchronize()
 
 
+def test_outer_step_in_a_cuda_graph(oracle):
+    """The steady-state outer step with overlap_steps = 1 launches one kernel whose arguments do
+    not change from step to step, so it can be captured once and replayed (small fragments are
+    launch-bound).  The host-side counters advance at capture time only; the replays must still
+    equal the oracle step for step."""
+    M, P = 4, 50_001
+    st, _ = make(M, P, 1550, 0, guards=False)
+    h = host_copy(st)
+    state = binding.State.from_dict(st)
+    stream = torch.cuda.Stream(device=DEV)
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        state.outer_eager(stream=stream)                       # warm-up launch outside the capture (also a real step)
+        oracle_outer(oracle, 2, h, M, P, st["stride"], 0.7, 0.9, 0)
+        stream.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            state.outer_eager(stream=stream)
+    for k in range(3):
+        inputs.inner_phase_standin(st)
+        h["theta"] = to_numpy(st["theta"])
+        graph.replay()
+        torch.cuda.synchronize()
+        oracle_outer(oracle, 2, h, M, P, st["stride"], 0.7, 0.9, 0)
+        assert_state_equal(st, h, what=f"graph replay {k + 1}")
+    assert state.get_counters()[1] == 2                        # the warm-up and the captured call; replays count nothing
+    state.close()
+
+
 def test_non_default_stream(oracle):
     M, P = 4, 100_001
     st, _ = make(M, P, 1500, 0)
