@@ -181,3 +181,27 @@ def test_a_fragment_step_touches_only_its_fragment_and_schedules_commute(oracle)
     b = run(sorted(schedule, key=lambda tf: (tf[1], tf[0])))
     for key in ("start", "outer_mom", "delta_prev_local", "delta_prev_avg"):
         np.testing.assert_array_equal(a[key], b[key], err_msg=key)
+
+
+def test_quantised_fragment_takes_its_scale_from_the_fragment(oracle):
+    """A fragment is what one exchange carries, so its EXMY scale is the maximum over the
+    fragment's own indices: the step equals the whole-vector quantised step of the slice taken on
+    its own, and differs from a step whose scale came from a larger outer gradient elsewhere."""
+    rng = np.random.default_rng(77)
+    D, M, P = 1, 2, 96
+    st = _frag_state(rng, D, M, P)
+    st["theta"][0, 80] = st["start"][0, 80] - 1.0             # a huge outer gradient outside the fragment [0, 64)
+    a = {k: v.copy() for k, v in st.items()}
+    oracle.outer_step_fragment(2, 0, 1, 0, 64, M=M, eta=0.7, mu=0.9, comm=oracle.COMM_EXMY, exp_bits=2, man_bits=1, **a)
+    b = {k: np.ascontiguousarray(v[..., :64]) for k, v in st.items()}
+    oracle.outer_step(2, M=M, P=64, stride=64, eta=0.7, mu=0.9, comm=oracle.COMM_EXMY, exp_bits=2, man_bits=1,
+                      theta=b["theta"], start=b["start"], outer_mom=b["outer_mom"],
+                      delta_prev_local=b["delta_prev_local"][0], delta_prev_avg=b["delta_prev_avg"][0])
+    for key in a:
+        np.testing.assert_array_equal(a[key][..., :64], b[key], err_msg=key)
+        np.testing.assert_array_equal(a[key][..., 64:], st[key][..., 64:], err_msg=key)   # the rest untouched
+    c = {k: v.copy() for k, v in st.items()}
+    oracle.outer_step(2, M=M, P=P, stride=P, eta=0.7, mu=0.9, comm=oracle.COMM_EXMY, exp_bits=2, man_bits=1,
+                      theta=c["theta"], start=c["start"], outer_mom=c["outer_mom"],
+                      delta_prev_local=c["delta_prev_local"][0], delta_prev_avg=c["delta_prev_avg"][0])
+    assert not np.array_equal(c["delta_prev_avg"][0, :64], a["delta_prev_avg"][0, :64])   # the whole-vector scale is coarser
