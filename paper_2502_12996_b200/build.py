@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libdiloco.so"
 REPORT = PKG / "ptxas_report.txt"        # registers / spills of every kernel, written by each build
-OUTER_M = [0, 1, 2, 3, 4, 8, 16, 1000, 1002, 1003]   # translation units: replica counts with kernels of their own, the
+OUTER_M = [0, 1, 2, 3, 4, 8, 16, 1000, 1002, 1003, 1004]   # translation units: replica counts with kernels of their own, the
                                                  # warp-split forms (1000, 1002) and the first-steps form (0)
 OBJ = PKG / "_obj"
 

@@ -145,7 +145,8 @@ int split_shape_for(int M, int forced) {
   if (forced == DILOCO_IMPL_SPLIT_R2 && M <= 32) return SHAPE_SPLIT_R2; // 16 warps per block at most
   if (forced == DILOCO_IMPL_SPLIT_R4) return SHAPE_SPLIT_R4;
   if (M <= 20) return SHAPE_SPLIT_R2;
-  return M <= 48 ? SHAPE_SPLIT_R4 : SHAPE_SPLIT_R8;
+  if (M <= 40) return SHAPE_SPLIT_R4;
+  return M <= 48 ? SHAPE_SPLIT_R6 : SHAPE_SPLIT_R8; // blocks of at most 8 warps beyond M = 40
 }
 
 template <bool Q>
@@ -167,6 +168,7 @@ int launch_outer_direct(const diloco_state *st, int var, bool boot, const OuterA
   switch (split_shape_for(M, impl)) {
     case SHAPE_SPLIT_R2: return launch_outer_shape<SHAPE_SPLIT_R2, Q>(var, tk, a, s);
     case SHAPE_SPLIT_R8: return launch_outer_shape<SHAPE_SPLIT_R8, Q>(var, tk, a, s);
+    case SHAPE_SPLIT_R6: return launch_outer_shape<SHAPE_SPLIT_R6, Q>(var, tk, a, s);
     default: return launch_outer_shape<SHAPE_SPLIT_R4, Q>(var, tk, a, s);
   }
 }

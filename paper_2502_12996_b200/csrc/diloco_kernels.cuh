@@ -679,7 +679,7 @@ __global__ void __launch_bounds__(NT, MINB) outer_step_chain_kernel(const OuterA
 // elements of every row: at least 1 KB per row and block measured 3 % faster than 512 bytes
 // (the DRAM pages a block opens are used more fully).  Shared memory GROUPS x M x V x 32 floats.
 template <int VAR, int TK, bool Q, int V, int R>
-__global__ void __launch_bounds__(R <= 4 ? 512 : 256, 2) outer_step_split_kernel(const OuterArgs a) {
+__global__ void __launch_bounds__(R <= 4 ? 512 : 256, R == 6 ? 3 : 2) outer_step_split_kernel(const OuterArgs a) {
   extern __shared__ float sent_all[];  // [groups][M][V][32]
   const int wpg = a.wpg;               // warps per group: one group = all M replicas of 32 columns
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;

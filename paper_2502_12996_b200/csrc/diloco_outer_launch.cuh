@@ -117,12 +117,14 @@ int launch_outer_first_steps(int var, int tk, const OuterArgs &a, cudaStream_t s
 //                   (6.55-6.8 TB/s at M = 5 .. 20; one replica per warp measured 5.8-6.2 at
 //                   M = 5, 6, 7 and 4.4-5.6 beyond), SPLIT_R4 four per warp with 64-bit accesses
 //                   above (6.5 TB/s at M = 24, 32 against 6.1-6.3 for R2: blocks of more than 10
-//                   warps wait too long at the barrier), SPLIT_R8 eight per warp above M = 48
-//                   (M = 64: 6.44 against 5.9 TB/s, blocks of 8 warps instead of 16); two column
+//                   warps wait too long at the barrier), SPLIT_R6 six per warp for M = 41 .. 48
+//                   and SPLIT_R8 eight per warp above (blocks of at most 8 warps: M = 44 6.50
+//                   against 5.85 TB/s, M = 64 6.44 against 5.9; seven per warp for M = 49 .. 56
+//                   measured no better than eight: 6.0-6.3); two column
 //                   groups per block where that keeps the SM's thread slots filled
 // The ID names a translation unit: a replica count with its own kernels (1, 2, 3, 4, 8, 16), one
 // of the split forms, or the first-steps form.
-enum { SHAPE_FIRST_STEPS = 0, SHAPE_SPLIT_R4 = 1000, SHAPE_SPLIT_R2 = 1002, SHAPE_SPLIT_R8 = 1003 };
+enum { SHAPE_FIRST_STEPS = 0, SHAPE_SPLIT_R4 = 1000, SHAPE_SPLIT_R2 = 1002, SHAPE_SPLIT_R8 = 1003, SHAPE_SPLIT_R6 = 1004 };
 
 template <int ID, bool Q>
 int launch_outer_shape(int var, int tk, const OuterArgs &a, cudaStream_t s) {
@@ -137,10 +139,11 @@ int launch_outer_shape(int var, int tk, const OuterArgs &a, cudaStream_t s) {
   else if constexpr (ID == SHAPE_SPLIT_R4) return launch_outer_split<Q, 2, 4>(var, tk, a, s);
   else if constexpr (ID == SHAPE_SPLIT_R2) return launch_outer_split<Q, 4, 2>(var, tk, a, s);
   else if constexpr (ID == SHAPE_SPLIT_R8) return launch_outer_split<Q, 2, 8>(var, tk, a, s);
+  else if constexpr (ID == SHAPE_SPLIT_R6) return launch_outer_split<Q, 2, 6>(var, tk, a, s);
   else return launch_outer_first_steps<Q>(var, tk, a, s);
 }
 
 // the translation units
-#define DILOCO_FOR_EACH_SHAPE(X) X(0) X(1) X(2) X(3) X(4) X(8) X(1000) X(1002) X(1003) X(16)
+#define DILOCO_FOR_EACH_SHAPE(X) X(0) X(1) X(2) X(3) X(4) X(8) X(1000) X(1002) X(1003) X(1004) X(16)
 
 } // namespace diloco
