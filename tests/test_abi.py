@@ -135,3 +135,12 @@ def test_no_kernel_spills_registers(lib):
     assert len(res) > 100
     bad = [(n, r, s, st) for n, r, s, st in res if s > 0 or st > 0]
     assert not bad, bad
+
+
+def test_header_is_plain_c():
+    """The boundary is a C ABI: the header must compile as C99 on its own (no C++, no CUDA types)."""
+    import subprocess
+    for cmd in (["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-fsyntax-only", "-x", "c", str(HEADER)],
+                ["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", str(HEADER)]):
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        assert res.returncode == 0, res.stderr
